@@ -1,0 +1,468 @@
+"""Pins of the CPU oracle against things other than itself.
+
+Each test fixes the oracle to a value the paper, the mathematics or an
+independent library fixes: cuRAND's host Philox generator, a separate NumPy
+restatement of Philox, closed forms, brute force in extended precision,
+torch's float64 cross-entropy, finite differences of the Assistant objective,
+and the literal sequential loop of Algorithm 1.
+"""
+import ctypes
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import aa_oracle as O
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "closed_forms.txt")
+
+
+def golden():
+    out = {}
+    for line in open(GOLDEN):
+        line = line.strip()
+        if line and not line.startswith("#"):
+            k, v = line.split()
+            out[k] = float(v)
+    return out
+
+
+# --------------------------------------------------------------------------
+# Philox4x32-10
+# --------------------------------------------------------------------------
+
+def _curand():
+    for path in ("/usr/local/cuda/lib64/libcurand.so.10", "libcurand.so.10", "libcurand.so"):
+        try:
+            return ctypes.CDLL(path)
+        except OSError:
+            continue
+    try:
+        import nvidia.curand
+
+        base = os.path.join(os.path.dirname(nvidia.curand.__file__), "lib")
+        for f in os.listdir(base):
+            if f.startswith("libcurand.so"):
+                return ctypes.CDLL(os.path.join(base, f))
+    except Exception:
+        pass
+    return None
+
+
+def _curand_words(lib, seed, offset, n):
+    gen = ctypes.c_void_p()
+    assert lib.curandCreateGeneratorHost(ctypes.byref(gen), 161) == 0  # CURAND_RNG_PSEUDO_PHILOX4_32_10
+    assert lib.curandSetPseudoRandomGeneratorSeed(gen, ctypes.c_ulonglong(seed)) == 0
+    assert lib.curandSetGeneratorOffset(gen, ctypes.c_ulonglong(offset)) == 0
+    out = np.zeros(n, dtype=np.uint32)
+    assert lib.curandGenerate(gen, out.ctypes.data_as(ctypes.c_void_p), ctypes.c_size_t(n)) == 0
+    lib.curandDestroyGenerator(gen)
+    return out
+
+
+@pytest.mark.parametrize("seed", [0, 1, 0x9F3A5C7E12345678])
+@pytest.mark.parametrize("block", [0, 3, (1 << 32) + 5])
+def test_philox_matches_curand_host_generator(seed, block):
+    """cuRAND's host generator: seed -> key; in its default ordering output block q (four
+    words) comes from subsequence q mod 65536 (counter words 2-3) at position q div 65536
+    (counter words 0-1), so one call pins the key and every counter position."""
+    lib = _curand()
+    if lib is None:
+        pytest.skip("libcurand not found")
+    words = _curand_words(lib, seed, 4 * block * 65536, 32)
+    key = [seed & 0xFFFFFFFF, seed >> 32]
+    for sub in range(8):
+        ref = O.philox4x32_10([block & 0xFFFFFFFF, block >> 32, sub, 0], key)
+        assert [int(v) for v in ref] == [int(v) for v in words[4 * sub:4 * sub + 4]]
+
+
+def _philox_numpy(ctr, key):
+    """Independent vectorised restatement (uint64 arithmetic) of Philox4x32-10."""
+    c = [np.asarray(v, dtype=np.uint64) for v in ctr]
+    k = [np.asarray(v, dtype=np.uint64) for v in key]
+    mask = np.uint64(0xFFFFFFFF)
+    for _ in range(10):
+        prod_a = np.uint64(0xD2511F53) * c[0]
+        prod_b = np.uint64(0xCD9E8D57) * c[2]
+        c = [((prod_b >> np.uint64(32)) ^ c[1] ^ k[0]) & mask, prod_b & mask,
+             ((prod_a >> np.uint64(32)) ^ c[3] ^ k[1]) & mask, prod_a & mask]
+        k = [(k[0] + np.uint64(0x9E3779B9)) & mask, (k[1] + np.uint64(0xBB67AE85)) & mask]
+    return [v.astype(np.uint32) for v in c]
+
+
+def test_philox_matches_numpy_restatement_on_all_counter_words():
+    rng = np.random.default_rng(11)
+    ctr = rng.integers(0, 1 << 32, size=(4, 256), dtype=np.uint64)
+    key = rng.integers(0, 1 << 32, size=(2, 256), dtype=np.uint64)
+    ref = _philox_numpy(list(ctr), list(key))
+    for t in range(256):
+        got = O.philox4x32_10(ctr[:, t], key[:, t])
+        assert [int(v) for v in got] == [int(ref[j][t]) for j in range(4)]
+
+
+def test_uniform_keying_and_range():
+    """c = top 24 bits of word 0 at counter (id, step), key = seed."""
+    seed, step = 0x0123456789ABCDEF, (7 << 32) + 3
+    ids = np.array([0, 1, 5, (1 << 32) + 9], dtype=np.uint64)
+    u = O.uniform(seed, step, ids)
+    for i, ui in zip(ids, u):
+        i = int(i)
+        words = _philox_numpy([i & 0xFFFFFFFF, i >> 32, step & 0xFFFFFFFF, step >> 32],
+                              [seed & 0xFFFFFFFF, seed >> 32])
+        assert ui == float(int(words[0]) >> 8) / float(1 << 24)
+        assert 0.0 <= ui < 1.0
+        assert np.float32(ui) == ui  # exact in fp32
+
+
+def test_uniform_statistics_and_stream_separation():
+    n = 200_000
+    ids = np.arange(n)
+    u0 = O.uniform(0, 0, ids)
+    u1 = O.uniform(0, 1, ids)
+    u2 = O.uniform(1, 0, ids)
+    for u in (u0, u1, u2):
+        assert abs(u.mean() - 0.5) < 5 * math.sqrt(1 / 12 / n)
+        assert abs(u.var() - 1 / 12) < 5 * math.sqrt(1 / 180 / n)
+        hist = np.bincount((u * 256).astype(int), minlength=256)
+        chi2 = ((hist - n / 256) ** 2 / (n / 256)).sum()
+        assert chi2 < 255 + 6 * math.sqrt(2 * 255)
+    lim = 5 / math.sqrt(n)
+    assert abs(np.corrcoef(u0[:-1], u0[1:])[0, 1]) < lim   # across ids
+    assert abs(np.corrcoef(u0, u1)[0, 1]) < lim            # across steps
+    assert abs(np.corrcoef(u0, u2)[0, 1]) < lim            # across seeds
+
+
+# --------------------------------------------------------------------------
+# Scores, g, acceptance probability
+# --------------------------------------------------------------------------
+
+def test_zero_weights_give_the_closed_form_probability():
+    x = np.random.default_rng(0).standard_normal((37, 19)).astype(np.float32)
+    s = O.score_dense(x, np.zeros(19, np.float32), 0.0)
+    assert np.all(s == 0.0)
+    g = O.sigmoid(s)
+    assert np.all(g == 0.5)
+    gold = golden()
+    for gamma in (0.1, 0.2, 0.05, 0.5):
+        assert np.allclose(O.accept_prob(g, gamma), gold[f"accept_prob_zero_weights_gamma_{gamma}"], atol=1e-15)
+
+
+def test_score_is_the_inner_product_one_hot_and_bias():
+    d = 23
+    w = np.random.default_rng(1).standard_normal(d).astype(np.float32)
+    x = np.eye(d, dtype=np.float32)
+    s = O.score_dense(x, w, 0.25)
+    assert np.array_equal(s, w.astype(np.float64) + 0.25)
+    # a wrong stride or transposed operand fails this: non-square, distinct entries
+    x2 = np.arange(3 * d, dtype=np.float32).reshape(3, d) / 7
+    expect = [math.fsum(float(a) * float(b) for a, b in zip(row, w)) - 1.5 for row in x2]
+    assert np.allclose(O.score_dense(x2, w, -1.5), expect, rtol=1e-14, atol=1e-12)
+    # gather list
+    assert np.array_equal(O.score_dense(x2, w, 0.0, row_idx=[2, 0]), O.score_dense(x2, w, 0.0)[[2, 0]])
+
+
+def test_bf16_rows_are_widened_exactly():
+    t = torch.tensor([[1.0, -2.5, 0.33203125], [3.0, 0.0078125, -0.5]], dtype=torch.bfloat16)
+    bits = t.view(torch.int16).numpy().view(np.uint16)
+    w = np.array([2.0, 4.0, 8.0], np.float32)
+    assert np.array_equal(O.score_dense(bits, w, 0.0), (t.double().numpy() * w).sum(1))
+
+
+def test_csr_score_equals_dense_score_with_duplicates():
+    rng = np.random.default_rng(2)
+    n, d = 41, 30
+    dense = np.zeros((n, d), np.float32)
+    indptr, col, val = [0], [], []
+    for i in range(n):
+        k = int(rng.integers(0, 9))        # empty rows included
+        cols = rng.integers(0, d, k)       # duplicates allowed
+        vals = rng.integers(1, 4, k).astype(np.float32)
+        for c, v in zip(cols, vals):
+            dense[i, c] += v
+        col += list(cols); val += list(vals); indptr.append(len(col))
+    w = rng.standard_normal(d).astype(np.float32)
+    a = O.score_csr(indptr, np.array(col, np.int32), np.array(val, np.float32), w, 0.5)
+    b = O.score_dense(dense, w, 0.5)
+    assert np.allclose(a, b, rtol=1e-13, atol=1e-13)
+
+
+def test_sigmoid_symmetry_and_extremes():
+    s = np.array([-800.0, -30.0, -1.0, 0.0, 1.0, 30.0, 800.0])
+    g = O.sigmoid(s)
+    assert np.all(np.isfinite(g)) and g[0] == 0.0 and g[-1] == 1.0 and g[3] == 0.5
+    assert np.allclose(g + g[::-1], 1.0, atol=1e-16)
+    assert np.allclose(g[4], 1 / (1 + math.exp(-1.0)), rtol=1e-15)
+
+
+def test_mlp_score_reduces_to_known_cases():
+    rng = np.random.default_rng(3)
+    n, d = 9, 6
+    x = rng.standard_normal((n, d)).astype(np.float32)
+    # selector W1 = I, w2 = 1: s = sum_j relu(x_j)
+    s = O.score_mlp(x, np.eye(d), np.zeros(d), np.ones(d), 0.0)
+    assert np.allclose(s, np.maximum(x.astype(np.float64), 0).sum(1), rtol=1e-15)
+    # one hidden unit, positive inputs and weights: equals the linear score scaled by w2
+    xp = np.abs(x) + 0.1
+    w = np.abs(rng.standard_normal(d)) + 0.1
+    s1 = O.score_mlp(xp.astype(np.float32), w[None, :], np.array([0.3]), np.array([2.0]), -1.0)
+    assert np.allclose(s1, 2.0 * (O.score_dense(xp.astype(np.float32), w, 0.3)) - 1.0, rtol=1e-14)
+    # non-square W1 with distinct entries against explicit loops (catches a transposed W1)
+    W1 = rng.standard_normal((4, d)); b1 = rng.standard_normal(4); w2 = rng.standard_normal(4)
+    s2, a2 = O.score_mlp(x, W1, b1, w2, 0.7, want_pre=True)
+    for i in range(n):
+        pre = [math.fsum(W1[u, j] * float(x[i, j]) for j in range(d)) + b1[u] for u in range(4)]
+        assert np.allclose(a2[i], pre, rtol=1e-13, atol=1e-13)
+        assert math.isclose(s2[i], 0.7 + sum(w2[u] * max(pre[u], 0.0) for u in range(4)), rel_tol=1e-12, abs_tol=1e-12)
+
+
+# --------------------------------------------------------------------------
+# Algorithm 1: shrink decision and ordered batch
+# --------------------------------------------------------------------------
+
+def test_two_branch_rule_equals_single_compare_away_from_ties():
+    rng = np.random.default_rng(4)
+    n = 50_000
+    g = rng.random(n)
+    for gamma in (0.0, 0.05, 0.1, 0.2, 0.5, 0.9):
+        keep = O.shrink(g, gamma, seed=3, step=9)
+        c = O.uniform(3, 9, np.arange(n))
+        p = O.accept_prob(g, gamma)
+        far = np.abs(c - p) > 1e-12
+        assert np.array_equal(keep[far].astype(bool), (c < p)[far])
+
+
+def test_gamma_extremes():
+    n = 5000
+    g = np.random.default_rng(5).random(n)
+    assert np.all(O.shrink(g, 1.0, 0, 0) == 1)                          # floor accepts everything
+    assert np.array_equal(O.compact(O.shrink(g, 1.0, 0, 0)), np.arange(n, dtype=np.int32))
+    c = O.uniform(0, 0, np.arange(n))
+    assert np.array_equal(O.shrink(g, 0.0, 0, 0).astype(bool), c < g)   # pure Bernoulli(g)
+    assert np.all(O.shrink(np.ones(n), 0.0, 0, 0) == 1)                 # p = 1 always keeps (c < 1)
+    assert np.all(O.shrink(np.zeros(n), 0.0, 0, 0) == 0)                # p = 0 never keeps
+
+
+def test_acceptance_count_is_consistent_with_the_probabilities():
+    rng = np.random.default_rng(6)
+    n = 100_000
+    g = O.sigmoid(rng.standard_normal(n) * 2)
+    for gamma, step in ((0.1, 0), (0.2, 1), (0.5, 2)):
+        p = O.accept_prob(g, gamma)
+        keep = O.shrink(g, gamma, 0, step)
+        sd = math.sqrt((p * (1 - p)).sum())
+        assert abs(keep.sum() - p.sum()) < 5 * sd
+        # calibration per decile of p
+        order = np.argsort(p)
+        for chunk in np.array_split(order, 10):
+            sdc = math.sqrt((p[chunk] * (1 - p[chunk])).sum())
+            assert abs(keep[chunk].sum() - p[chunk].sum()) < 5 * sdc
+
+
+def test_compaction_is_nonzero_of_the_mask_in_order():
+    rng = np.random.default_rng(7)
+    for n in (0, 1, 2, 31, 32, 33, 1000):
+        keep = (rng.random(n) < 0.4).astype(np.uint8)
+        B = O.compact(keep)
+        assert np.array_equal(B, np.nonzero(keep)[0].astype(np.int32))
+        assert len(B) == int(keep.sum())
+        assert np.all(np.diff(B) > 0)
+    perm = rng.permutation(1000).astype(np.int32)
+    keep = (rng.random(1000) < 0.4).astype(np.uint8)
+    assert np.array_equal(O.compact(keep, row_idx=perm), perm[np.nonzero(keep)[0]])
+
+
+def test_sequential_algorithm_1_is_a_prefix_of_the_ordered_survivors():
+    rng = np.random.default_rng(8)
+    n = 4000
+    g = rng.random(n)
+    perm = rng.permutation(n).astype(np.int32)
+    for row_idx in (None, perm):
+        full = O.compact(O.shrink(g, 0.15, 21, 4, id_base=100, row_idx=row_idx), row_idx=row_idx)
+        for bs in (1, 7, 64, len(full), len(full) + 50):
+            B, consumed = O.sample_batch(g, 0.15, 21, 4, bs, id_base=100, row_idx=row_idx)
+            assert np.array_equal(B, full[:bs])
+            if bs <= len(full):
+                rows = perm if row_idx is not None else np.arange(n)
+                assert rows[consumed - 1] == full[bs - 1]   # stopped right after the bs-th accept
+            else:
+                assert consumed == n
+
+
+# --------------------------------------------------------------------------
+# Boss loss per instance
+# --------------------------------------------------------------------------
+
+@pytest.mark.parametrize("C", [1, 2, 10, 100, 1000, 32000])
+def test_uniform_logits_give_ln_C(C):
+    logits = np.full((3, C), 1.75, np.float32)
+    ell = O.row_loss(logits, np.array([0, C // 2, C - 1], np.int32))
+    assert np.allclose(ell, math.log(C), rtol=0, atol=1e-12)
+
+
+def test_row_loss_against_long_double_brute_force():
+    rng = np.random.default_rng(9)
+    logits = (rng.standard_normal((64, 13)) * 2).astype(np.float32)
+    labels = rng.integers(0, 13, 64).astype(np.int32)
+    ell = O.row_loss(logits, labels)
+    ld = logits.astype(np.longdouble)
+    brute = np.log(np.exp(ld).sum(1)) - ld[np.arange(64), labels]
+    assert np.allclose(ell, brute.astype(np.float64), rtol=0, atol=1e-13)
+
+
+def test_row_loss_matches_torch_float64_cross_entropy():
+    rng = np.random.default_rng(10)
+    logits = (rng.standard_normal((200, 77)) * 4).astype(np.float32)
+    labels = rng.integers(0, 77, 200).astype(np.int32)
+    ref = torch.nn.functional.cross_entropy(torch.from_numpy(logits).double(),
+                                            torch.from_numpy(labels).long(), reduction="none").numpy()
+    assert np.allclose(O.row_loss(logits, labels), ref, rtol=0, atol=1e-12)
+    # bf16 storage: same check on the widened values
+    t = torch.from_numpy(logits).to(torch.bfloat16)
+    ref16 = torch.nn.functional.cross_entropy(t.double(), torch.from_numpy(labels).long(), reduction="none").numpy()
+    assert np.allclose(O.row_loss(t.view(torch.int16).numpy().view(np.uint16), labels), ref16, rtol=0, atol=1e-12)
+
+
+def test_row_loss_properties():
+    rng = np.random.default_rng(12)
+    logits = (rng.standard_normal((50, 9)) * 3).astype(np.float32)
+    labels = rng.integers(0, 9, 50).astype(np.int32)
+    base = O.row_loss(logits, labels)
+    assert np.allclose(O.row_loss(logits + np.float32(8.0), labels), base, atol=1e-5)   # shift invariance
+    # two classes: softplus of the gap
+    two = np.array([[0.3, -1.2], [2.0, 5.0]], np.float32)
+    assert np.allclose(O.row_loss(two, [0, 0]), [math.log1p(math.exp(-1.5)), math.log1p(math.exp(3.0))], atol=1e-7)
+    # dominant logit: ~0 when it is the label, ~gap otherwise
+    dom = np.zeros((2, 6), np.float32); dom[:, 2] = 60.0
+    out = O.row_loss(dom, [2, 4])
+    assert out[0] < 1e-20 + 1e-12 and abs(out[1] - 60.0) < 1e-12
+    # huge magnitudes stay finite (max subtraction), -inf entries are masked
+    big = np.array([[1e30, -1e30, 0.0], [-np.inf, 0.0, 0.0]], np.float32)
+    out = O.row_loss(big, [0, 1])
+    assert out[0] == 0.0 and abs(out[1] - math.log(2)) < 1e-15
+    # padding (negative label) and out-of-range labels contribute 0
+    assert np.array_equal(O.row_loss(logits[:2], [-1, 9]), [0.0, 0.0])
+
+
+def test_segment_sums():
+    rng = np.random.default_rng(13)
+    ell = rng.random(40)
+    assert np.array_equal(O.segment_sum(ell, np.arange(41)), ell)                      # identity offsets
+    assert math.isclose(O.segment_sum(ell, [0, 40])[0], math.fsum(ell), rel_tol=1e-14)  # one segment
+    off = [0, 3, 3, 17, 40]                                                            # empty segment -> 0
+    L = O.segment_sum(ell, off)
+    assert L[1] == 0.0
+    assert np.allclose(L, [math.fsum(ell[a:b]) for a, b in zip(off[:-1], off[1:])], rtol=1e-14)
+    assert math.isclose(L.sum(), math.fsum(ell), rel_tol=1e-13)                        # additivity
+
+
+# --------------------------------------------------------------------------
+# Labels, objective, gradient, update
+# --------------------------------------------------------------------------
+
+def test_label_rule_is_strict_and_batch_mean():
+    gold = golden()
+    f = np.full(100, 2.5, np.float32)
+    assert O.labels(f, O.batch_mean(f)).sum() == gold["labels_constant_loss_positive_count"]
+    f2 = np.array([1.0, 3.0, 1.0, 3.0, 3.0], np.float32)
+    assert O.batch_mean(f2) == 2.2
+    assert np.array_equal(O.labels(f2, O.batch_mean(f2)), [0, 1, 0, 1, 1])
+    assert np.array_equal(O.labels(f2, 3.0), [0, 0, 0, 0, 0])     # f > T, not >=
+    assert O.batch_mean(np.zeros(0, np.float32)) == 0.0
+
+
+def test_objective_closed_forms():
+    gold = golden()
+    z = np.array([0, 1, 1, 0, 1], np.uint8)
+    assert math.isclose(O.bce_mean(np.zeros(5), z), gold["bce_zero_weights"], rel_tol=1e-15)
+    s = np.array([0.7, -1.3, 2.0, 12.0, -12.0])   # the direct form below loses g = 1 beyond |s| ~ 36
+    g = 1 / (1 + np.exp(-s))
+    direct = -(z * np.log(g) + (1 - z) * np.log1p(-g)).mean()
+    assert math.isclose(O.bce_mean(s, z), direct, rel_tol=1e-10)
+    # far tails: BCE -> |s| on the wrong side, 0 on the right side
+    assert math.isclose(O.bce_mean(np.array([800.0, -800.0, 800.0]), np.array([0, 1, 1], np.uint8)), 1600.0 / 3)
+
+
+def _fd(fun, theta, h=1e-6):
+    out = np.zeros_like(theta)
+    flat, of = theta.reshape(-1), out.reshape(-1)
+    for j in range(flat.size):
+        keep = flat[j]
+        flat[j] = keep + h; up = fun()
+        flat[j] = keep - h; dn = fun()
+        flat[j] = keep
+        of[j] = (up - dn) / (2 * h)
+    return out
+
+
+def test_linear_gradient_matches_finite_differences_dense_and_csr():
+    rng = np.random.default_rng(14)
+    m, d = 17, 7
+    x = rng.standard_normal((m + 3, d)).astype(np.float32)
+    rows = rng.permutation(m + 3)[:m].astype(np.int32)
+    z = rng.integers(0, 2, m).astype(np.uint8)
+    w = rng.standard_normal(d) * 0.5
+    bb = np.array([0.2])
+    obj = lambda: O.bce_mean(O.score_dense(x, w, bb[0], row_idx=rows), z)
+    gw, gb = O.linear_grad_dense(x, O.score_dense(x, w, bb[0], row_idx=rows), z, row_idx=rows)
+    assert np.allclose(gw, _fd(obj, w), rtol=1e-6, atol=1e-9)
+    assert np.allclose(gb, _fd(obj, bb)[0], rtol=1e-6, atol=1e-9)
+    # CSR with duplicate columns
+    indptr, col, val = [0], [], []
+    for i in range(m):
+        k = int(rng.integers(0, 6)); col += list(rng.integers(0, d, k)); val += list(rng.random(k) + 0.5)
+        indptr.append(len(col))
+    col, val = np.array(col, np.int32), np.array(val, np.float32)
+    obj2 = lambda: O.bce_mean(O.score_csr(indptr, col, val, w, bb[0]), z)
+    gw2, gb2 = O.linear_grad_csr(indptr, col, val, d, O.score_csr(indptr, col, val, w, bb[0]), z)
+    assert np.allclose(gw2, _fd(obj2, w), rtol=1e-6, atol=1e-9)
+    assert np.allclose(gb2, _fd(obj2, bb)[0], rtol=1e-6, atol=1e-9)
+
+
+def test_mlp_gradient_matches_finite_differences():
+    rng = np.random.default_rng(15)
+    m, d, hdim = 11, 5, 4
+    x = rng.standard_normal((m, d)).astype(np.float32)
+    z = rng.integers(0, 2, m).astype(np.uint8)
+    W1 = rng.standard_normal((hdim, d)) * 0.7
+    b1 = rng.standard_normal(hdim) * 0.3
+    w2 = rng.standard_normal(hdim)
+    b2 = np.array([0.1])
+    obj = lambda: O.bce_mean(O.score_mlp(x, W1, b1, w2, b2[0]), z)
+    s, a = O.score_mlp(x, W1, b1, w2, b2[0], want_pre=True)
+    assert np.min(np.abs(a)) > 1e-4   # no unit sits on the ReLU kink within the FD step
+    gW1, gb1, gw2, gb2 = O.mlp_grad(x, a, s, z, w2)
+    assert np.allclose(gW1, _fd(obj, W1), rtol=1e-6, atol=1e-9)
+    assert np.allclose(gb1, _fd(obj, b1), rtol=1e-6, atol=1e-9)
+    assert np.allclose(gw2, _fd(obj, w2), rtol=1e-6, atol=1e-9)
+    assert np.allclose(gb2, _fd(obj, b2)[0], rtol=1e-6, atol=1e-9)
+
+
+def test_update_special_cases():
+    # one instance, x = e_j: only w_j and b move, by -lr (sigma(w_j + b) - z)
+    d, j = 6, 4
+    w = np.linspace(-0.5, 0.5, d).astype(np.float32)
+    b = np.float32(0.25)
+    x = np.zeros((1, d), np.float32); x[0, j] = 1.0
+    f = np.array([5.0], np.float32)
+    w1, b1, z = O.assistant_step_linear_dense(x, f, w, b, lr=0.5, T=1.0)
+    assert z[0] == 1
+    delta = -0.5 * (1 / (1 + math.exp(-(float(w[j]) + 0.25))) - 1.0)
+    expect = w.copy(); expect[j] = np.float32(float(w[j]) + delta)
+    assert np.array_equal(w1, expect)
+    assert b1 == np.float32(0.25 + delta)
+    # lr = 0 and empty batch leave the parameters unchanged
+    w2, b2, _ = O.assistant_step_linear_dense(x, f, w, b, lr=0.0, T=1.0)
+    assert np.array_equal(w2, w) and b2 == b
+    w3, b3, _ = O.assistant_step_linear_dense(x, np.zeros(0, np.float32), w, b, lr=0.5)
+    assert np.array_equal(w3, w) and b3 == b
+
+
+def test_bf16_rounding_is_nearest_even():
+    src = np.array([1.0, 1.00390625, 1.01171875, -3.0e-41, 3.3895314e38, np.inf], np.float32)
+    ref = torch.from_numpy(src).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(O.round_bf16(src), ref)
+    rnd = np.random.default_rng(16).standard_normal(10000).astype(np.float32)
+    ref = torch.from_numpy(rnd).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(O.round_bf16(rnd), ref)
