@@ -1,0 +1,367 @@
+"""Throughput of the instance-shrinking batch generator on the image-classification shape.
+
+One step = one pass of the whole hot path over one candidate pool: Assistant score ->
+Bernoulli shrink -> ordered batch list (aa_score_shrink), per-instance Boss loss of the
+accepted batch (aa_instance_loss), labels + one Assistant SGD step (aa_assistant_step).
+Pool: 65,536 candidates x 3072 bf16 features (403 MB, larger than L2; pools rotate),
+100-class fp32 logits, gamma 0.1, lr 0.05.  Prints ONE JSON line on rank 0.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+N > 1 is launched with torch.distributed.run, one rank per GPU; every rank screens its own
+pools with its own Assistant (the path shards by instance, no data-path collective), and the
+reported value is all ranks' candidates over the slowest rank's device time.
+--impl reference times the CPU oracle (as it stands) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "candidates screened/sec (score+shrink+compact -> instance loss -> Assistant step)"
+UNIT = "candidates/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--pools", type=int, default=8, help="distinct resident pools rotated through the steps")
+    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--cpu-steps", type=int, default=4, help="oracle steps timed for cpu_baseline (0 = skip)")
+    ap.add_argument("--pool-rows", type=int, default=None, help="override the pool size (testing only)")
+    return ap.parse_args()
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def ncu_traffic_bytes():
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if still valid."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        with open(path) as f:
+            rec = json.load(f)
+        return rec.get("score_shrink_dense_bf16_n65536_d3072_dram_bytes_per_launch")
+    except Exception:
+        return None
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------
+# CPU oracle leg (cpu_baseline and --impl reference)
+# --------------------------------------------------------------------------
+
+def oracle_step_seconds(cfg, x_host, w0, logits_host, labels_host, steps: int):
+    """Times `steps` whole steps of the oracle, as it stands, single-threaded.  Returns (seconds, candidates)."""
+    import numpy as np
+
+    from oracle import aa_oracle as O
+
+    w, b = w0.copy(), np.float32(0.0)
+    n = x_host.shape[0]
+    t0 = time.perf_counter()
+    for step in range(steps):
+        scr = O.screen_linear_dense(x_host, w, b, cfg.gamma, cfg.philox_seed, step)
+        Bidx = scr["B"]
+        m = len(Bidx)
+        f = O.row_loss(logits_host[:m], labels_host[:m]).astype(np.float32)
+        w, b, _ = O.assistant_step_linear_dense(x_host, f, w, b, cfg.lr, row_idx=Bidx)
+    return time.perf_counter() - t0, n * steps
+
+
+def run_reference(args, cfg):
+    """The reference arm: the CPU oracle on this machine's host cores, bounded sample per step."""
+    import torch
+
+    from oracle import aa_oracle as O
+    from paper_1905_03381_b200 import workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    O.build()
+    sample_rows = min(cfg.n, 8192)
+    x = W.to_oracle(W.uniform01((sample_rows, cfg.d), 100, torch.bfloat16, "cpu"))
+    w0 = W.linear_assistant(cfg.d, 2, "cpu")[0].numpy()
+    logits = W.normal((sample_rows, cfg.classes), 3.0, 200, torch.float32, "cpu").numpy()
+    labels = W.randint(0, cfg.classes, (sample_rows,), 300, "cpu").numpy()
+    for _ in range(min(args.warmup, 2)):
+        oracle_step_seconds(cfg, x, w0, logits, labels, 1)
+    steps = max(1, min(args.steps, 16))
+    sec, cand = oracle_step_seconds(cfg, x, w0, logits, labels, steps)
+    value = cand / sec
+    sample = f"{sample_rows} of {cfg.n} candidates per step, {steps} steps"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": min(args.warmup, 2), "ms_per_step": 1e3 * sec / steps * (cfg.n / sample_rows),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(cfg, args, reference=True),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(cfg, args, reference=False):
+    return {
+        "workload": "image-classification shape: pool 65,536 x 3072 bf16 features U[0,1), linear Assistant, "
+                    "100-class fp32 logits N(0,3), mix 0.1, SGD lr 0.05 every step",
+        "pool_rows": cfg.n, "d": cfg.d, "classes": cfg.classes, "mix": cfg.gamma, "lr": cfg.lr,
+        "pools_rotated": None if reference else args.pools,
+        "l2_policy": "inputs larger than L2: each pool is 403 MB and pools rotate",
+        "parallelism": f"instance-sharded x{args.gpus}, one Assistant per GPU, no data-path collective",
+    }
+
+
+# --------------------------------------------------------------------------
+# GPU arm
+# --------------------------------------------------------------------------
+
+def run_b200(args, cfg):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    from paper_1905_03381_b200 import binding as B, build as lib_build, sharding, workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU path (use --impl reference for the oracle)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        lib_build.build()
+    if world > 1:
+        dist.barrier()
+
+    plan = sharding.plan(rank, world, args.pools, cfg.n)
+    pools = [cfg.pool(pid, dev) for pid in plan.pool_ids]
+    logits = [cfg.logits(pid, dev) for pid in plan.pool_ids]
+    labels = [cfg.labels(pid, dev) for pid in plan.pool_ids]
+    w, b = cfg.assistant(dev)
+    aa = B.AutoAssist(max_rows=cfg.n, max_d=cfg.d, device=dev)
+    asst = B.linear_assistant(w, b)
+    out_idx = torch.zeros(cfg.n, dtype=torch.int32, device=dev)
+    out_count = torch.zeros(1, dtype=torch.int32, device=dev)
+    loss = torch.zeros(cfg.n, dtype=torch.float32, device=dev)
+    feats = [B.dense_features(p, id_base=base) for p, base in zip(pools, plan.id_bases)]
+    batch_feats = [B.dense_features(p, row_idx=out_idx, id_base=base) for p, base in zip(pools, plan.id_bases)]
+    lg = [B.logits_desc(l) for l in logits]
+    npool = len(pools)
+
+    def step(i, events=None):
+        k = i % npool
+        if events is not None:
+            events[0].record()
+        aa.aa_score_shrink(feats[k], asst, cfg.gamma, cfg.philox_seed, i, out_idx, out_count)
+        if events is not None:
+            events[1].record()
+        aa.aa_instance_loss(lg[k], labels[k], loss, count_dev=out_count)
+        if events is not None:
+            events[2].record()
+        aa.aa_assistant_step(batch_feats[k], loss, asst, cfg.lr, count_dev=out_count)
+        if events is not None:
+            events[3].record()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+    assert aa.aa_device_status() == B.AA_OK
+
+    # ---- device-resident throughput: K steps between two events, kernels timed per call as well
+    K = args.steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = aa.aa_launch_count()
+    accepted = 0
+    barrier()
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for i in range(K):
+        step(args.warmup + i, ev[i])
+    t_end.record()
+    barrier()
+    elapsed_ms = t_start.elapsed_time(t_end)
+    launches = aa.aa_launch_count() - launches0
+    if rank == 0:
+        time.sleep(0.2)
+        sampler.stop()
+    status = aa.aa_device_status()
+    assert status == B.AA_OK, B.status_string(status)
+    accepted = int(out_count.item())
+    score_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / K
+    loss_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / K
+    asst_ms = sum(e[2].elapsed_time(e[3]) for e in ev) / K
+
+    agg = sharding.aggregate(dist if world > 1 else None, dev, elapsed_ms, cfg.n * K)
+
+    # ---- end to end through the host-buffer entry point (pinned host inputs, results read back)
+    e2e = None
+    if args.e2e_steps > 0:
+        xh = pools[0].cpu().pin_memory()
+        lh = logits[0].cpu().pin_memory()
+        yh = labels[0].cpu().pin_memory()
+        idx_h = torch.zeros(cfg.n, dtype=torch.int32).pin_memory()
+        cnt_h = torch.zeros(1, dtype=torch.int32).pin_memory()
+        loss_h = torch.zeros(cfg.n, dtype=torch.float32).pin_memory()
+        hf, hl, staging, sbytes = aa.host_step_plan(xh, lh)
+        for i in range(3):
+            aa.aa_step_host(hf, asst, cfg.gamma, cfg.philox_seed, i, hl, yh, cfg.lr, idx_h, cnt_h, loss_h, staging, sbytes)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        d2h = 0
+        for i in range(args.e2e_steps):
+            aa.aa_step_host(hf, asst, cfg.gamma, cfg.philox_seed, 1000 + i, hl, yh, cfg.lr, idx_h, cnt_h, loss_h, staging, sbytes)
+            d2h += 4 + 8 * int(cnt_h.item())
+        e1.record()
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
+        e2e_agg = sharding.aggregate(dist if world > 1 else None, dev, e2e_ms, cfg.n * args.e2e_steps)
+        h2d = xh.numel() * xh.element_size() + lh.numel() * lh.element_size() + yh.numel() * yh.element_size()
+        e2e = {"value": e2e_agg["units"] / (e2e_agg["ms"] * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h // args.e2e_steps, "steps": args.e2e_steps,
+               "ms_per_step": e2e_agg["ms"] / args.e2e_steps}
+        del xh, lh, yh, staging
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak_gbs()
+    alg_bytes = cfg.n * cfg.d * 2 + cfg.d * 4 + accepted * 4 + 4
+    achieved = alg_bytes / (score_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "score_shrink_dense_kernel<bf16>", "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": ncu_traffic_bytes(),
+                "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": score_ms,
+                "frac_of_nominal_8TBs": achieved / 8000.0}
+    loss_bytes = accepted * (cfg.classes * 4 + 8)
+    asst_bytes = accepted * (cfg.d * 2 + 8) + 2 * cfg.d * 4
+    stages = {
+        "score_shrink": {"ms": score_ms, "GB/s": achieved},
+        "instance_loss": {"ms": loss_ms, "GB/s": loss_bytes / (loss_ms * 1e-3) / 1e9, "rows_per_s": accepted / (loss_ms * 1e-3)},
+        "assistant_step": {"ms": asst_ms, "GB/s": asst_bytes / (asst_ms * 1e-3) / 1e9},
+    }
+
+    cpu = None
+    if world == 1 and args.cpu_steps > 0:
+        from oracle import aa_oracle as O
+        O.build()
+        xs = W.to_oracle(pools[0])
+        w0 = cfg.assistant("cpu")[0].numpy()
+        sec, cand = oracle_step_seconds(cfg, xs, w0, logits[0].cpu().numpy(), labels[0].cpu().numpy(), args.cpu_steps)
+        cpu = {"value": cand / sec, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": f"{args.cpu_steps} whole steps on one full pool of {cfg.n} candidates ({sec:.1f} s)"}
+
+    line = {
+        "metric": METRIC, "value": agg["units"] / (agg["ms"] * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+        "warmup": max(args.warmup, 3), "ms_per_step": agg["ms"] / K, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(cfg, args),
+        "roofline": roofline, "stages": stages, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
+        "accepted_last_step": accepted, "clocks": sampler.summary(),
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    from paper_1905_03381_b200 import workloads as W
+
+    cfg = W.ImageShape()
+    if args.pool_rows:
+        cfg.n = args.pool_rows
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_b200(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,190 @@
+// Internal declarations shared by the kernels of the AutoAssist batch-generator library.
+// Nothing here is part of the C ABI (that is include/autoassist.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "autoassist.h"
+
+namespace aa {
+
+// Device-resident control block at the start of the caller's workspace.
+struct Control {
+    unsigned int ticket;   // next tile to hand out (dynamic tile order = look-back order)
+    unsigned int done;     // CTAs of the running scan kernel that have finished
+    unsigned int epoch;    // generation of the look-back flags; bumped by the last CTA of each scan
+    int status;            // first device-side condition latched (aa_status), 0 = none
+    unsigned int pad[60];
+};
+static_assert(sizeof(Control) == 256, "control block is one 256-byte line group");
+
+constexpr int kMaxTileRows = 1024;     // rows of one compaction tile (multiple of 32)
+constexpr int kScanThreads = 128;      // CTA size of the score/shrink/compact kernels
+constexpr int kMaxParts = 1024;        // upper bound on per-CTA gradient partials
+constexpr unsigned kSpinLimit = 1u << 22;   // polls before a look-back wait gives up
+
+struct aa_ctx_impl {
+    char* ws;
+    size_t ws_bytes;
+    cudaStream_t stream;
+    int device;
+    int sm_count;
+    int64_t max_rows, max_d, max_hidden;
+    Control* ctl;
+    unsigned long long* tile_state;   // one packed (flag, value) word per tile
+    int64_t max_tiles;
+    float* row_scratch;               // max_rows floats: row losses / residuals
+    float* partials;                  // gradient partial sums
+    int64_t partial_floats;
+    int64_t launches;
+    uint64_t scans_since_clear;
+};
+
+// Arguments of the shrink + compaction tail shared by every scoring front end.
+struct ShrinkParams {
+    Control* ctl;
+    unsigned long long* tile_state;
+    int64_t n_cand;          // candidates in the pool
+    int64_t n_stored;        // stored rows (bound for row_idx entries)
+    const int32_t* row_idx;  // optional candidate list
+    int64_t id_base;
+    float mix;               // gamma of Algorithm 1
+    uint32_t seed_lo, seed_hi, step_lo, step_hi;
+    int32_t* out_idx;
+    int64_t capacity;
+    int32_t* out_count;
+    float* out_score;
+    uint8_t* out_mask;
+    int tile_rows;
+    unsigned int n_tiles;
+};
+
+// ---------------------------------------------------------------- device helpers
+#ifdef __CUDACC__
+
+__device__ __forceinline__ void latch(Control* ctl, int code) { atomicCAS(&ctl->status, 0, code); }
+
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float lg2_approx(float x) {
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// g = sigmoid(s) without overflow on either side.
+__device__ __forceinline__ float sigmoid_f32(float s) {
+    float e = expf(-fabsf(s));
+    float pos = 1.0f / (1.0f + e);
+    return s >= 0.0f ? pos : e * pos;
+}
+
+// Philox4x32-10 (Salmon et al., SC'11); returns output word 0 only.
+__device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                         uint32_t k0, uint32_t k1) {
+#pragma unroll
+    for (int round = 0; round < 10; ++round) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        c0 = hi1 ^ c1 ^ k0;
+        c1 = lo1;
+        c2 = hi0 ^ c3 ^ k1;
+        c3 = lo0;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    return c0;
+}
+
+// The uniform draw c of Algorithm 1 for instance `id` at `step`: 24 random bits scaled to [0, 1).
+__device__ __forceinline__ float philox_uniform(const ShrinkParams& p, uint64_t id) {
+    const uint32_t w = philox4x32_10_word0((uint32_t)id, (uint32_t)(id >> 32), p.step_lo, p.step_hi, p.seed_lo, p.seed_hi);
+    return (float)(w >> 8) * (1.0f / 16777216.0f);
+}
+
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t packed) { return __uint_as_float(packed << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t packed) { return __uint_as_float(packed & 0xFFFF0000u); }
+
+// 16-byte vector of stored elements widened to fp32.
+template <typename T>
+struct Vec;
+template <>
+struct Vec<float> {
+    static constexpr int kElems = 4;
+    __device__ static __forceinline__ void unpack(const uint4& v, float (&out)[4]) {
+        out[0] = __uint_as_float(v.x); out[1] = __uint_as_float(v.y);
+        out[2] = __uint_as_float(v.z); out[3] = __uint_as_float(v.w);
+    }
+    __device__ static __forceinline__ void load(const float* p, float (&out)[4]) {
+        unpack(__ldg(reinterpret_cast<const uint4*>(p)), out);
+    }
+    __device__ static __forceinline__ float one(const float* p) { return __ldg(p); }
+};
+template <>
+struct Vec<uint16_t> {   // bf16 bit patterns
+    static constexpr int kElems = 8;
+    __device__ static __forceinline__ void unpack(const uint4& v, float (&out)[8]) {
+        out[0] = bf16_lo(v.x); out[1] = bf16_hi(v.x);
+        out[2] = bf16_lo(v.y); out[3] = bf16_hi(v.y);
+        out[4] = bf16_lo(v.z); out[5] = bf16_hi(v.z);
+        out[6] = bf16_lo(v.w); out[7] = bf16_hi(v.w);
+    }
+    __device__ static __forceinline__ void load(const uint16_t* p, float (&out)[8]) {
+        unpack(__ldg(reinterpret_cast<const uint4*>(p)), out);
+    }
+    __device__ static __forceinline__ float one(const uint16_t* p) { return __uint_as_float((uint32_t)__ldg(p) << 16); }
+};
+
+#endif  // __CUDACC__
+
+// ---------------------------------------------------------------- host-side launchers (one per .cu)
+struct DenseFeat {
+    const void* base;
+    int dtype;
+    int64_t d, row_stride;
+    const float* w;
+    const float* b;
+};
+struct CsrFeat {
+    const int32_t* indptr;
+    const int32_t* col;
+    const float* val;
+    int64_t d;
+    const float* w;
+    const float* b;
+    float mean_nnz;
+};
+
+aa_status launch_score_shrink_dense(aa_ctx_impl* c, const DenseFeat& f, ShrinkParams sp);
+aa_status launch_score_shrink_csr(aa_ctx_impl* c, const CsrFeat& f, ShrinkParams sp);
+aa_status launch_shrink_from_scores(aa_ctx_impl* c, const float* score, ShrinkParams sp);
+
+aa_status launch_instance_loss(aa_ctx_impl* c, const aa_logits& lg, const int32_t* labels, const int32_t* offsets,
+                               int64_t n_seg, const int32_t* count_dev, float* out_loss);
+
+aa_status launch_assistant_step_dense(aa_ctx_impl* c, const DenseFeat& f, const int32_t* row_idx, int64_t n_stored,
+                                      int64_t m_host, const int32_t* count_dev, const float* loss, float* w, float* b,
+                                      float lr, int thresh_mode, float threshold);
+aa_status launch_assistant_step_csr(aa_ctx_impl* c, const CsrFeat& f, const int32_t* row_idx, int64_t n_stored,
+                                    int64_t m_host, const int32_t* count_dev, const float* loss, float* w, float* b,
+                                    float lr, int thresh_mode, float threshold);
+
+// Persistent-grid size for a kernel: CTAs that fit on the device at once.
+int resident_ctas(aa_ctx_impl* c, const void* kernel, int threads, size_t dyn_smem);
+
+inline aa_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? AA_OK : AA_ERR_CUDA; }
+
+}  // namespace aa

@@ -1,0 +1,396 @@
+// Assistant labels + one SGD step (Sec. 5.2 label rule and objective; Algorithm 2:
+// Assistant.gradient, Assistant.update) for the linear Assistant g = sigmoid(w.x + b).
+//
+// Dense features: each CTA stages a block of batch rows in shared memory once, computes
+// their residuals r_i = g_i - z_i (one warp per row) and then adds r_i x_i into column
+// accumulators that stay in registers for the whole kernel (each thread owns fixed
+// columns).  CTAs write their column sums to a partial buffer; a second small kernel adds
+// the partials in a fixed order and applies  w <- w - lr * grad,  so the result does not
+// depend on scheduling.  CSR features: residuals first, then a scatter of -lr/M r_i val
+// onto the touched weights with fp32 atomics.
+#include <math.h>
+
+#include "aa_internal.cuh"
+
+namespace aa {
+
+namespace {
+
+constexpr int kStepThreads = 512;
+constexpr int kStepWarps = kStepThreads / 32;
+
+struct StepParams {
+    DenseFeat f;
+    CsrFeat csr;
+    const int32_t* row_idx;
+    int64_t n_stored;
+    int64_t m_host;
+    const int32_t* count_dev;
+    const float* loss;
+    int thresh_mode;
+    float threshold;
+    float lr;
+    float* w;
+    float* b;
+    float* partials;      // [parts][d_pad] column sums, then [parts] bias sums
+    float* residual;      // per batch row (CSR path)
+    int64_t d_pad;
+    int rows_per_block;
+    Control* ctl;
+};
+
+__device__ __forceinline__ int64_t batch_size(const StepParams& p) {
+    int64_t m = p.m_host;
+    if (p.count_dev) {
+        const int64_t c = *p.count_dev;
+        m = c < 0 ? 0 : (c < m ? c : m);
+    }
+    return m;
+}
+
+// Shrinking threshold T: the caller's value, or the mean of the batch losses.  Every CTA adds the
+// losses in the same order (fp64), so all CTAs agree on T bit for bit.
+__device__ double block_threshold(const StepParams& p, int64_t m, double* red /* [warps] */) {
+    if (p.thresh_mode == AA_THRESH_VALUE) return (double)p.threshold;
+    double acc = 0.0;
+    for (int64_t i = threadIdx.x; i < m; i += blockDim.x) acc += (double)__ldg(p.loss + i);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    if (lane == 0) red[warp] = acc;
+    __syncthreads();
+    double total = 0.0;
+    for (int wi = 0; wi < nwarps; ++wi) total += red[wi];
+    __syncthreads();
+    return m > 0 ? total / (double)m : 0.0;
+}
+
+__device__ __forceinline__ long long batch_row(const StepParams& p, int64_t i) {
+    if (!p.row_idx) return i;
+    const long long r = p.row_idx[i];
+    if ((unsigned long long)r >= (unsigned long long)p.n_stored) {
+        latch(p.ctl, AA_ERR_BAD_INDEX);
+        return -1;
+    }
+    return r;
+}
+
+// ---------------------------------------------------------------- dense
+// CI = 16-byte column vectors owned by each thread.  VEC = rows are 16-byte aligned.
+template <typename T, int CI, bool VEC>
+__global__ void __launch_bounds__(kStepThreads) linear_grad_dense_kernel(StepParams p) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    constexpr int VE = Vec<T>::kElems;
+    __shared__ double red[kStepWarps];
+    __shared__ float res[32];              // residual per staged row
+    float* w_s = reinterpret_cast<float*>(smem_raw);                 // [d_pad]
+    T* x_s = reinterpret_cast<T*>(smem_raw + p.d_pad * sizeof(float));   // [rows_per_block][d_pad]
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int64_t d = p.f.d, d_pad = p.d_pad;
+    const int nvec = (int)(d_pad / VE);
+    const int RB = p.rows_per_block;
+    const int64_t m = batch_size(p);
+    const double T_shrink = block_threshold(p, m, red);
+
+    for (int64_t j = tid; j < d_pad; j += kStepThreads) w_s[j] = j < d ? p.f.w[j] : 0.0f;
+    const float bias = *p.f.b;
+    const T* base = static_cast<const T*>(p.f.base);
+
+    float acc[CI][VE];
+#pragma unroll
+    for (int ci = 0; ci < CI; ++ci)
+#pragma unroll
+        for (int e = 0; e < VE; ++e) acc[ci][e] = 0.0f;
+    float bias_acc = 0.0f;   // used by lane 0 of each warp
+
+    const int64_t n_blocks = (m + RB - 1) / RB;
+    for (int64_t blk = blockIdx.x; blk < n_blocks; blk += gridDim.x) {
+        const int64_t i0 = blk * RB;
+        __syncthreads();   // previous block's readers are done (and w_s is complete)
+        // stage the rows
+        if (VEC) {
+            for (int q = tid; q < RB * nvec; q += kStepThreads) {
+                const int rl = q / nvec, v = q - rl * nvec;
+                const int64_t i = i0 + rl;
+                uint4 val = make_uint4(0, 0, 0, 0);
+                if (i < m) {
+                    const long long r = batch_row(p, i);
+                    if (r >= 0) val = __ldg(reinterpret_cast<const uint4*>(base + r * p.f.row_stride) + v);
+                }
+                reinterpret_cast<uint4*>(x_s + (int64_t)rl * d_pad)[v] = val;
+            }
+        } else {
+            for (int64_t q = tid; q < (int64_t)RB * d_pad; q += kStepThreads) {
+                const int rl = (int)(q / d_pad);
+                const int64_t j = q - (int64_t)rl * d_pad;
+                const int64_t i = i0 + rl;
+                T val = T(0);
+                if (i < m && j < d) {
+                    const long long r = batch_row(p, i);
+                    if (r >= 0) val = base[r * p.f.row_stride + j];
+                }
+                x_s[(int64_t)rl * d_pad + j] = val;
+            }
+        }
+        __syncthreads();
+        // residuals, one warp per staged row
+        for (int rl = warp; rl < RB; rl += kStepWarps) {
+            const int64_t i = i0 + rl;
+            float dot = 0.0f;
+            const T* xr = x_s + (int64_t)rl * d_pad;
+            for (int v = lane; v < nvec; v += 32) {
+                float x[VE];
+                Vec<T>::unpack(reinterpret_cast<const uint4*>(xr)[v], x);
+                const float* wp = w_s + (int64_t)v * VE;
+#pragma unroll
+                for (int e = 0; e < VE; ++e) dot = fmaf(x[e], wp[e], dot);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, o);
+            if (lane == 0) {
+                float r = 0.0f;
+                if (i < m) {
+                    const float z = (double)__ldg(p.loss + i) > T_shrink ? 1.0f : 0.0f;
+                    r = sigmoid_f32(dot + bias) - z;
+                    if (p.row_idx && (unsigned long long)(long long)p.row_idx[i] >= (unsigned long long)p.n_stored) r = 0.0f;
+                    bias_acc += r;
+                }
+                res[rl] = r;
+            }
+        }
+        __syncthreads();
+        // column sums: acc += r_i * x_i
+#pragma unroll
+        for (int ci = 0; ci < CI; ++ci) {
+            const int v = tid + ci * kStepThreads;
+            if (v < nvec) {
+                for (int rl = 0; rl < RB; ++rl) {
+                    const float r = res[rl];
+                    float x[VE];
+                    Vec<T>::unpack(reinterpret_cast<const uint4*>(x_s + (int64_t)rl * d_pad)[v], x);
+#pragma unroll
+                    for (int e = 0; e < VE; ++e) acc[ci][e] = fmaf(r, x[e], acc[ci][e]);
+                }
+            }
+        }
+    }
+
+    // this CTA's column sums and bias sum
+    float* part = p.partials + (int64_t)blockIdx.x * d_pad;
+#pragma unroll
+    for (int ci = 0; ci < CI; ++ci) {
+        const int v = tid + ci * kStepThreads;
+        if (v < nvec) {
+#pragma unroll
+            for (int e = 0; e < VE; ++e) part[(int64_t)v * VE + e] = acc[ci][e];
+        }
+    }
+    __syncthreads();
+    float* bred = reinterpret_cast<float*>(red);
+    if (lane == 0) bred[warp] = bias_acc;
+    __syncthreads();
+    if (tid == 0) {
+        float t = 0.0f;
+        for (int wi = 0; wi < kStepWarps; ++wi) t += bred[wi];
+        p.partials[(int64_t)gridDim.x * d_pad + blockIdx.x] = t;
+    }
+}
+
+// Adds the partials in CTA order and applies the SGD update.
+__global__ void __launch_bounds__(256) linear_apply_kernel(StepParams p, int parts) {
+    const int64_t m = batch_size(p);
+    if (m <= 0) return;
+    const float scale = p.lr / (float)m;
+    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j < p.f.d) {
+        float g = 0.0f;
+        for (int q = 0; q < parts; ++q) g += p.partials[(int64_t)q * p.d_pad + j];
+        p.w[j] = p.w[j] - scale * g;
+    }
+    if (j == 0) {
+        float g = 0.0f;
+        for (int q = 0; q < parts; ++q) g += p.partials[(int64_t)parts * p.d_pad + q];
+        p.b[0] = p.b[0] - scale * g;
+    }
+}
+
+// ---------------------------------------------------------------- CSR
+template <int LPR>
+__global__ void __launch_bounds__(256) csr_residual_kernel(StepParams p) {
+    __shared__ double red[8];
+    const int64_t m = batch_size(p);
+    const double T_shrink = block_threshold(p, m, red);
+    const float bias = *p.csr.b;
+    const int gl = threadIdx.x % LPR;
+    const int64_t groups = (int64_t)gridDim.x * (blockDim.x / LPR);
+    const int64_t g0 = (int64_t)blockIdx.x * (blockDim.x / LPR) + threadIdx.x / LPR;
+    const int64_t rounds = (m + groups - 1) / groups;
+    for (int64_t it = 0; it < rounds; ++it) {
+        const int64_t i = g0 + it * groups;
+        const long long r = i < m ? batch_row(p, i) : -1;
+        float acc = 0.0f;
+        if (r >= 0) {
+            const int e0 = __ldg(p.csr.indptr + r), e1 = __ldg(p.csr.indptr + r + 1);
+            for (int e = e0 + gl; e < e1; e += LPR) {
+                const int c = __ldg(p.csr.col + e);
+                if ((unsigned long long)(unsigned int)c < (unsigned long long)p.csr.d) acc = fmaf(__ldg(p.csr.val + e), p.w[c], acc);
+                else latch(p.ctl, AA_ERR_BAD_INDEX);
+            }
+        }
+#pragma unroll
+        for (int o = LPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+        if (gl == 0 && i < m) {
+            float res = 0.0f;
+            if (r >= 0) {
+                const float z = (double)__ldg(p.loss + i) > T_shrink ? 1.0f : 0.0f;
+                res = sigmoid_f32(acc + bias) - z;
+            }
+            p.residual[i] = res;
+        }
+    }
+}
+
+template <int LPR>
+__global__ void __launch_bounds__(256) csr_scatter_kernel(StepParams p) {
+    const int64_t m = batch_size(p);
+    if (m <= 0) return;
+    const float scale = -p.lr / (float)m;
+    const int gl = threadIdx.x % LPR;
+    const int64_t groups = (int64_t)gridDim.x * (blockDim.x / LPR);
+    const int64_t g0 = (int64_t)blockIdx.x * (blockDim.x / LPR) + threadIdx.x / LPR;
+    const int64_t rounds = (m + groups - 1) / groups;
+    float bias_acc = 0.0f;
+    for (int64_t it = 0; it < rounds; ++it) {
+        const int64_t i = g0 + it * groups;
+        if (i >= m) continue;
+        const long long r = p.row_idx ? (long long)p.row_idx[i] : i;
+        if ((unsigned long long)r >= (unsigned long long)p.n_stored) continue;   // latched by the residual pass
+        const float step = scale * p.residual[i];
+        if (gl == 0) bias_acc += step;
+        const int e0 = __ldg(p.csr.indptr + r), e1 = __ldg(p.csr.indptr + r + 1);
+        for (int e = e0 + gl; e < e1; e += LPR) {
+            const int c = __ldg(p.csr.col + e);
+            if ((unsigned long long)(unsigned int)c < (unsigned long long)p.csr.d) atomicAdd(p.w + c, step * __ldg(p.csr.val + e));
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) bias_acc += __shfl_xor_sync(0xFFFFFFFFu, bias_acc, o);
+    if ((threadIdx.x & 31) == 0 && bias_acc != 0.0f) atomicAdd(p.b, bias_acc);
+}
+
+template <typename T, bool VEC>
+const void* pick_dense_kernel(int ci) {
+    switch (ci) {
+        case 1: return (const void*)linear_grad_dense_kernel<T, 1, VEC>;
+        case 2: return (const void*)linear_grad_dense_kernel<T, 2, VEC>;
+        case 4: return (const void*)linear_grad_dense_kernel<T, 4, VEC>;
+        default: return (const void*)linear_grad_dense_kernel<T, 8, VEC>;
+    }
+}
+
+}  // namespace
+
+aa_status launch_assistant_step_dense(aa_ctx_impl* c, const DenseFeat& f, const int32_t* row_idx, int64_t n_stored,
+                                      int64_t m_host, const int32_t* count_dev, const float* loss, float* w, float* b,
+                                      float lr, int thresh_mode, float threshold) {
+    if (m_host <= 0) return AA_OK;
+    const int es = f.dtype == AA_BF16 ? 2 : 4;
+    const int ve = 16 / es;
+    const bool vec = ((uintptr_t)f.base % 16 == 0) && ((f.row_stride * es) % 16 == 0) && (f.d % ve == 0);
+    StepParams p = {};
+    p.f = f;
+    p.row_idx = row_idx;
+    p.n_stored = n_stored;
+    p.m_host = m_host;
+    p.count_dev = count_dev;
+    p.loss = loss;
+    p.thresh_mode = thresh_mode;
+    p.threshold = threshold;
+    p.lr = lr;
+    p.w = w;
+    p.b = b;
+    p.partials = c->partials;
+    p.ctl = c->ctl;
+    p.d_pad = (f.d + ve - 1) / ve * ve;
+    const int64_t nvec = p.d_pad / ve;
+    int ci = 1;
+    while (ci < 8 && (int64_t)ci * kStepThreads < nvec) ci <<= 1;
+    if ((int64_t)ci * kStepThreads < nvec) return AA_ERR_UNSUPPORTED;   // dense rows beyond 4096 vectors
+
+    // rows staged per block: as many as fit in ~64 KB beside w, between 1 and 32
+    const int64_t row_bytes = p.d_pad * es;
+    int64_t rb = (64 * 1024) / row_bytes;
+    rb = rb < 1 ? 1 : (rb > 32 ? 32 : rb);
+    p.rows_per_block = (int)rb;
+    const size_t smem = (size_t)p.d_pad * sizeof(float) + (size_t)rb * row_bytes;
+    if (smem > 200 * 1024) return AA_ERR_UNSUPPORTED;
+
+    const void* kernel = f.dtype == AA_BF16 ? (vec ? pick_dense_kernel<uint16_t, true>(ci) : pick_dense_kernel<uint16_t, false>(ci))
+                                            : (vec ? pick_dense_kernel<float, true>(ci) : pick_dense_kernel<float, false>(ci));
+    if (smem > 48 * 1024 &&
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return AA_ERR_CUDA;
+    int grid = resident_ctas(c, kernel, kStepThreads, smem);
+    if (grid <= 0) return AA_ERR_CUDA;
+    const int64_t n_blocks = (m_host + rb - 1) / rb;
+    if (grid > n_blocks) grid = (int)n_blocks;
+    const int64_t max_parts = c->partial_floats / (p.d_pad + 1);
+    if (max_parts < 1) return AA_ERR_WORKSPACE;
+    if (grid > max_parts) grid = (int)max_parts;
+    if (grid > kMaxParts) grid = kMaxParts;
+
+    void* args[] = {&p};
+    if (cudaLaunchKernel(kernel, dim3(grid), dim3(kStepThreads), args, smem, c->stream) != cudaSuccess) return AA_ERR_CUDA;
+    ++c->launches;
+    int parts = grid;
+    void* args2[] = {&p, &parts};
+    const int agrid = (int)((f.d + 255) / 256);
+    if (cudaLaunchKernel((const void*)linear_apply_kernel, dim3(agrid), dim3(256), args2, 0, c->stream) != cudaSuccess)
+        return AA_ERR_CUDA;
+    ++c->launches;
+    return AA_OK;
+}
+
+aa_status launch_assistant_step_csr(aa_ctx_impl* c, const CsrFeat& f, const int32_t* row_idx, int64_t n_stored,
+                                    int64_t m_host, const int32_t* count_dev, const float* loss, float* w, float* b,
+                                    float lr, int thresh_mode, float threshold) {
+    if (m_host <= 0) return AA_OK;
+    if (m_host > c->max_rows) return AA_ERR_WORKSPACE;
+    StepParams p = {};
+    p.csr = f;
+    p.row_idx = row_idx;
+    p.n_stored = n_stored;
+    p.m_host = m_host;
+    p.count_dev = count_dev;
+    p.loss = loss;
+    p.thresh_mode = thresh_mode;
+    p.threshold = threshold;
+    p.lr = lr;
+    p.w = w;
+    p.b = b;
+    p.residual = c->row_scratch;
+    p.ctl = c->ctl;
+    int lpr = 4;
+    while (lpr < 32 && lpr * 4 <= f.mean_nnz) lpr <<= 1;
+    const int64_t rows_per_cta = 256 / lpr;
+    const int64_t want = (m_host + rows_per_cta - 1) / rows_per_cta;
+    const int cap = c->sm_count * 8;
+    const int grid = (int)(want < cap ? want : cap);
+    void* args[] = {&p};
+    const void* k1;
+    const void* k2;
+    switch (lpr) {
+        case 4: k1 = (const void*)csr_residual_kernel<4>; k2 = (const void*)csr_scatter_kernel<4>; break;
+        case 8: k1 = (const void*)csr_residual_kernel<8>; k2 = (const void*)csr_scatter_kernel<8>; break;
+        case 16: k1 = (const void*)csr_residual_kernel<16>; k2 = (const void*)csr_scatter_kernel<16>; break;
+        default: k1 = (const void*)csr_residual_kernel<32>; k2 = (const void*)csr_scatter_kernel<32>; break;
+    }
+    if (cudaLaunchKernel(k1, dim3(grid), dim3(256), args, 0, c->stream) != cudaSuccess) return AA_ERR_CUDA;
+    ++c->launches;
+    if (cudaLaunchKernel(k2, dim3(grid), dim3(256), args, 0, c->stream) != cudaSuccess) return AA_ERR_CUDA;
+    ++c->launches;
+    return AA_OK;
+}
+
+}  // namespace aa

@@ -1,0 +1,276 @@
+// Per-instance Boss loss from logits (Sec. 5.3: the loss f pushed with each index i).
+//
+// Row cross-entropy  l_r = log sum_c exp(x_rc) - x_{r,y_r}  in a single pass over the row:
+// every thread keeps a running maximum M and a sum S of 2^(t - M) over its elements, with
+// t = x * log2(e), so that sum_c 2^(t_c) = S * 2^M; thread states are merged by warp shuffles
+// (and through shared memory when a CTA shares a row).  For sequence tasks the token rows of
+// a sentence are then summed in row order (fp64 accumulator) by a second small kernel.
+#include <math.h>
+
+#include "aa_internal.cuh"
+
+namespace aa {
+
+namespace {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr int kRowThreads = 256;   // CTA size when one CTA owns a row
+
+struct LossParams {
+    const void* logits;
+    int64_t rows, cols, row_stride;
+    const int32_t* labels;
+    const int32_t* count_dev;
+    float* out;
+    Control* ctl;
+};
+
+struct RunState {
+    float m;   // running maximum of t = x*log2(e)
+    float s;   // sum of 2^(t - m)
+};
+
+__device__ __forceinline__ void absorb(RunState& st, const float* t, int n) {
+    float vmax = t[0];
+    for (int e = 1; e < n; ++e) vmax = fmaxf(vmax, t[e]);
+    if (vmax > st.m) {
+        st.s *= ex2_approx(st.m - vmax);   // st.m = -inf gives 0 * 0
+        st.m = vmax;
+    }
+    const float ref = st.m == -INFINITY ? 0.0f : st.m;   // all -inf so far: every term is 2^-inf = 0
+    for (int e = 0; e < n; ++e) st.s += ex2_approx(t[e] - ref);
+}
+
+template <int N>
+__device__ __forceinline__ void absorb_vec(RunState& st, const float (&x)[N]) {
+    float t[N];
+#pragma unroll
+    for (int e = 0; e < N; ++e) t[e] = x[e] * kLog2e;
+    float vmax = t[0];
+#pragma unroll
+    for (int e = 1; e < N; ++e) vmax = fmaxf(vmax, t[e]);
+    if (vmax > st.m) {
+        st.s *= ex2_approx(st.m - vmax);
+        st.m = vmax;
+    }
+    const float ref = st.m == -INFINITY ? 0.0f : st.m;
+#pragma unroll
+    for (int e = 0; e < N; ++e) st.s += ex2_approx(t[e] - ref);
+}
+
+__device__ __forceinline__ RunState merge(const RunState& a, const RunState& b) {
+    RunState o;
+    o.m = fmaxf(a.m, b.m);
+    const float ref = o.m == -INFINITY ? 0.0f : o.m;
+    o.s = a.s * ex2_approx(a.m - ref) + b.s * ex2_approx(b.m - ref);
+    return o;
+}
+
+template <int WIDTH>
+__device__ __forceinline__ RunState group_merge(RunState st) {
+#pragma unroll
+    for (int o = WIDTH / 2; o > 0; o >>= 1) {
+        RunState other;
+        other.m = __shfl_xor_sync(0xFFFFFFFFu, st.m, o);
+        other.s = __shfl_xor_sync(0xFFFFFFFFu, st.s, o);
+        st = merge(st, other);
+    }
+    return st;
+}
+
+__device__ __forceinline__ float finish_row(const RunState& st, float label_logit) {
+    return (st.m + lg2_approx(st.s)) * kLn2 - label_logit;
+}
+
+__device__ __forceinline__ int64_t effective_rows(const LossParams& p) {
+    int64_t rows = p.rows;
+    if (p.count_dev) {
+        const int64_t c = *p.count_dev;
+        rows = c < 0 ? 0 : (c < rows ? c : rows);
+    }
+    return rows;
+}
+
+// Label of row r: >= 0 valid; -1 padding or invalid (invalid latches AA_ERR_BAD_INDEX).
+__device__ __forceinline__ int checked_label(const LossParams& p, int64_t r) {
+    const int y = __ldg(p.labels + r);
+    if (y < 0) return -1;
+    if (y >= p.cols) {
+        latch(p.ctl, AA_ERR_BAD_INDEX);
+        return -1;
+    }
+    return y;
+}
+
+// Accumulate the elements [j0, j1) of one row, strided over `nthreads` workers starting at `rank`.
+// Handles any alignment: scalar head up to the first 16-byte boundary, vector body, scalar tail.
+template <typename T>
+__device__ __forceinline__ void scan_row(RunState& st, const T* row, int64_t cols, int rank, int nthreads) {
+    constexpr int VE = Vec<T>::kElems;
+    const uintptr_t addr = (uintptr_t)row;
+    int64_t head = ((16 - (addr & 15)) & 15) / sizeof(T);
+    if (head > cols) head = cols;
+    const int64_t nvec = (cols - head) / VE;
+    const int64_t tail0 = head + nvec * VE;
+    const T* body = row + head;
+#pragma unroll 2
+    for (int64_t v = rank; v < nvec; v += nthreads) {
+        float x[VE];
+        Vec<T>::load(body + v * VE, x);
+        absorb_vec(st, x);
+    }
+    // the few unaligned elements at both ends
+    for (int64_t j = rank; j < head; j += nthreads) {
+        const float t = Vec<T>::one(row + j) * kLog2e;
+        absorb(st, &t, 1);
+    }
+    for (int64_t j = tail0 + rank; j < cols; j += nthreads) {
+        const float t = Vec<T>::one(row + j) * kLog2e;
+        absorb(st, &t, 1);
+    }
+}
+
+// Short rows: LPR lanes per row, several rows per warp.
+template <typename T, int LPR>
+__global__ void __launch_bounds__(256) row_loss_group_kernel(LossParams p) {
+    const int64_t rows = effective_rows(p);
+    const int gl = threadIdx.x % LPR;
+    const int64_t groups_per_grid = (int64_t)gridDim.x * (blockDim.x / LPR);
+    const int64_t group0 = (int64_t)blockIdx.x * (blockDim.x / LPR) + threadIdx.x / LPR;
+    // whole warps iterate together so that the shuffles see every lane
+    const int64_t rounds = (rows + groups_per_grid - 1) / groups_per_grid;
+    for (int64_t it = 0; it < rounds; ++it) {
+        const int64_t r = group0 + it * groups_per_grid;
+        RunState st = {-INFINITY, 0.0f};
+        int y = -1;
+        if (r < rows) {
+            y = checked_label(p, r);
+            if (y >= 0) scan_row<T>(st, static_cast<const T*>(p.logits) + r * p.row_stride, p.cols, gl, LPR);
+        }
+        st = group_merge<LPR>(st);
+        if (gl == 0 && r < rows) {
+            float loss = 0.0f;
+            if (y >= 0) loss = finish_row(st, Vec<T>::one(static_cast<const T*>(p.logits) + r * p.row_stride + y));
+            p.out[r] = loss;
+        }
+    }
+}
+
+// Long rows: one CTA per row.
+template <typename T>
+__global__ void __launch_bounds__(kRowThreads) row_loss_cta_kernel(LossParams p) {
+    __shared__ RunState warp_state[kRowThreads / 32];
+    const int64_t rows = effective_rows(p);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
+        const int y = checked_label(p, r);   // uniform over the CTA
+        if (y < 0) {
+            if (threadIdx.x == 0) p.out[r] = 0.0f;
+            continue;
+        }
+        const T* row = static_cast<const T*>(p.logits) + r * p.row_stride;
+        RunState st = {-INFINITY, 0.0f};
+        scan_row<T>(st, row, p.cols, threadIdx.x, kRowThreads);
+        st = group_merge<32>(st);
+        if (lane == 0) warp_state[warp] = st;
+        __syncthreads();
+        if (warp == 0) {
+            RunState t = lane < kRowThreads / 32 ? warp_state[lane] : RunState{-INFINITY, 0.0f};
+            t = group_merge<32>(t);
+            if (lane == 0) p.out[r] = finish_row(t, Vec<T>::one(row + y));
+        }
+        __syncthreads();
+    }
+}
+
+// Per-sentence sums of token-row losses, one warp per segment, rows added in fp64.
+__global__ void __launch_bounds__(256) segment_sum_kernel(const float* __restrict__ row_loss, const int32_t* __restrict__ offsets,
+                                                          int64_t n_seg, int64_t rows, float* __restrict__ out, Control* ctl) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t s = warp; s < n_seg; s += nwarps) {
+        const int64_t a = __ldg(offsets + s), b = __ldg(offsets + s + 1);
+        double acc = 0.0;
+        if (a < 0 || b < a || b > rows) {
+            if (lane == 0) latch(ctl, AA_ERR_BAD_INDEX);
+        } else {
+            for (int64_t r = a + lane; r < b; r += 32) acc += (double)row_loss[r];
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+        if (lane == 0) out[s] = (float)acc;
+    }
+}
+
+template <typename T>
+aa_status launch_rows(aa_ctx_impl* c, LossParams& p) {
+    const int es = (int)sizeof(T);
+    const int64_t row_bytes = p.cols * es;
+    void* args[] = {&p};
+    const void* kernel;
+    int threads, grid;
+    if (row_bytes >= 8 * 1024) {
+        kernel = (const void*)row_loss_cta_kernel<T>;
+        threads = kRowThreads;
+        int cap = resident_ctas(c, kernel, threads, 0);
+        if (cap <= 0) return AA_ERR_CUDA;
+        grid = (int)(p.rows < cap ? p.rows : cap);
+    } else {
+        const int64_t work = (row_bytes + 15) / 16;   // 16-byte vectors per row
+        int lpr = 2;
+        while (lpr < 32 && lpr * 4 <= work) lpr <<= 1;   // two to four vectors per lane
+        threads = 256;
+        switch (lpr) {
+            case 2: kernel = (const void*)row_loss_group_kernel<T, 2>; break;
+            case 4: kernel = (const void*)row_loss_group_kernel<T, 4>; break;
+            case 8: kernel = (const void*)row_loss_group_kernel<T, 8>; break;
+            case 16: kernel = (const void*)row_loss_group_kernel<T, 16>; break;
+            default: kernel = (const void*)row_loss_group_kernel<T, 32>; lpr = 32; break;
+        }
+        int cap = resident_ctas(c, kernel, threads, 0);
+        if (cap <= 0) return AA_ERR_CUDA;
+        const int64_t rows_per_cta = threads / lpr;
+        const int64_t want = (p.rows + rows_per_cta - 1) / rows_per_cta;
+        grid = (int)(want < cap ? want : cap);
+    }
+    if (grid < 1) grid = 1;
+    if (cudaLaunchKernel(kernel, dim3(grid), dim3(threads), args, 0, c->stream) != cudaSuccess) return AA_ERR_CUDA;
+    ++c->launches;
+    return AA_OK;
+}
+
+}  // namespace
+
+aa_status launch_instance_loss(aa_ctx_impl* c, const aa_logits& lg, const int32_t* labels, const int32_t* offsets,
+                               int64_t n_seg, const int32_t* count_dev, float* out_loss) {
+    LossParams p;
+    p.logits = lg.data;
+    p.rows = lg.rows;
+    p.cols = lg.cols;
+    p.row_stride = lg.row_stride;
+    p.labels = labels;
+    p.count_dev = offsets ? nullptr : count_dev;
+    p.ctl = c->ctl;
+    p.out = offsets ? c->row_scratch : out_loss;
+    if (lg.rows > 0) {
+        aa_status st = lg.dtype == AA_BF16 ? launch_rows<uint16_t>(c, p) : launch_rows<float>(c, p);
+        if (st != AA_OK) return st;
+    }
+    if (offsets && n_seg > 0) {
+        const float* row_loss = c->row_scratch;
+        int64_t rows = lg.rows;
+        Control* ctl = c->ctl;
+        void* args[] = {&row_loss, &offsets, &n_seg, &rows, &out_loss, &ctl};
+        const int64_t want = (n_seg + 7) / 8;   // 8 warps per CTA
+        const int cap = c->sm_count * 8;
+        const int grid = (int)(want < cap ? want : cap);
+        if (cudaLaunchKernel((const void*)segment_sum_kernel, dim3(grid), dim3(256), args, 0, c->stream) != cudaSuccess)
+            return AA_ERR_CUDA;
+        ++c->launches;
+    }
+    return AA_OK;
+}
+
+}  // namespace aa

@@ -1,0 +1,376 @@
+// Assistant score -> Bernoulli shrink -> ordered batch list, fused in one pass
+// (Algorithm 1, Assistant.sample_batch, evaluated for a whole candidate pool at once).
+//
+// Every kernel here is a persistent grid.  A CTA repeatedly takes the next tile of
+// candidates from a ticket counter, computes the tile's pre-activations, draws the
+// keep/skip decision per candidate (Philox keyed by seed, counter = (instance id,
+// step)), and appends the kept candidates to the batch list at the position given by a
+// decoupled look-back scan over the tiles, so that the list keeps candidate order.
+// Tiles are handed out in look-back order, so every tile a CTA waits on is owned by a
+// CTA that is already running; each wait is still bounded and gives up with a latched
+// AA_ERR_SCAN_TIMEOUT instead of spinning for ever.
+#include "aa_internal.cuh"
+
+namespace aa {
+
+namespace {
+
+struct TailSmem {
+    float s[kMaxTileRows];     // pre-activation per candidate of the tile
+    unsigned int mask[32];     // keep ballot per 32-candidate unit
+    int off[32];               // exclusive prefix of the unit counts inside the tile
+    int base;                  // kept candidates in all earlier tiles
+    unsigned int tile;
+};
+
+__device__ __forceinline__ unsigned long long pack_state(unsigned int flag, int value) {
+    return ((unsigned long long)flag << 32) | (unsigned int)value;
+}
+
+// Decoupled look-back (warp-collective, called by warp 0): publishes this tile's count and
+// returns the number kept in all earlier tiles.
+__device__ int lookback_exclusive(const ShrinkParams& p, unsigned int tile, unsigned int epoch, int total) {
+    const int lane = threadIdx.x & 31;
+    const unsigned int flag_agg = epoch * 4u + 1u, flag_inc = epoch * 4u + 2u;
+    unsigned long long* state = p.tile_state;
+    if (tile == 0) {
+        if (lane == 0) st_relaxed_u64(&state[0], pack_state(flag_inc, total));
+        return 0;
+    }
+    if (lane == 0) st_relaxed_u64(&state[tile], pack_state(flag_agg, total));
+    int excl = 0;
+    long long window_end = (long long)tile - 1;
+    bool gave_up = false;
+    while (!gave_up) {
+        const long long idx = window_end - lane;
+        unsigned int flag = flag_inc;   // lanes before tile 0 stand for "inclusive prefix 0"
+        int val = 0;
+        unsigned int polls = 0;
+        while (true) {
+            if (idx >= 0) {
+                const unsigned long long w = ld_relaxed_u64(&state[idx]);
+                flag = (unsigned int)(w >> 32);
+                val = (int)(unsigned int)w;
+            }
+            const unsigned int inc_m = __ballot_sync(0xFFFFFFFFu, flag == flag_inc);
+            const unsigned int agg_m = __ballot_sync(0xFFFFFFFFu, flag == flag_agg);
+            // only the tiles between this one and the nearest inclusive prefix have to be ready
+            const unsigned int need = inc_m ? ((1u << (__ffs(inc_m) - 1)) - 1u) : 0xFFFFFFFFu;
+            if (((inc_m | agg_m) & need) == need) break;
+            if (++polls > kSpinLimit) { gave_up = true; break; }
+            __nanosleep(polls < 64 ? 32 : 256);
+        }
+        if (gave_up) break;
+        const unsigned int inc_m = __ballot_sync(0xFFFFFFFFu, flag == flag_inc);
+        const int first = inc_m ? (__ffs(inc_m) - 1) : 31;
+        int contrib = lane <= first ? val : 0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) contrib += __shfl_xor_sync(0xFFFFFFFFu, contrib, o);
+        excl += contrib;
+        if (inc_m) break;
+        window_end -= 32;
+    }
+    if (gave_up && lane == 0) latch(p.ctl, AA_ERR_SCAN_TIMEOUT);
+    if (lane == 0) st_relaxed_u64(&state[tile], pack_state(flag_inc, excl + total));
+    return excl;
+}
+
+// Shrink decision + ordered append for one tile whose pre-activations are in sm.s.
+// All threads of the CTA call this; contains CTA barriers.
+__device__ void shrink_compact_tile(const ShrinkParams& p, unsigned int tile, unsigned int epoch, TailSmem& sm) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    const int units = p.tile_rows >> 5;
+    const long long k0 = (long long)tile * p.tile_rows;
+
+    for (int u = warp; u < units; u += nwarps) {
+        const long long k = k0 + u * 32 + lane;
+        bool keep = false;
+        if (k < p.n_cand) {
+            const float s = sm.s[u * 32 + lane];
+            const long long r = p.row_idx ? (long long)p.row_idx[k] : k;
+            // net acceptance probability of Algorithm 1: gamma + (1 - gamma) g
+            const float prob = fmaf(1.0f - p.mix, sigmoid_f32(s), p.mix);
+            const float c = philox_uniform(p, (uint64_t)(p.id_base + r));
+            keep = c < prob;   // false for the NaN that marks an unreadable row
+            if (p.out_score) p.out_score[k] = s;
+            if (p.out_mask) p.out_mask[k] = keep ? 1 : 0;
+        }
+        const unsigned int m = __ballot_sync(0xFFFFFFFFu, keep);
+        if (lane == 0) sm.mask[u] = m;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        const int cnt = lane < units ? __popc(sm.mask[lane]) : 0;
+        int inc = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+            if (lane >= o) inc += t;
+        }
+        sm.off[lane] = inc - cnt;
+        const int total = __shfl_sync(0xFFFFFFFFu, inc, 31);
+        const int base = lookback_exclusive(p, tile, epoch, total);
+        if (lane == 0) {
+            sm.base = base;
+            if (tile == p.n_tiles - 1) *p.out_count = base + total;
+        }
+    }
+    __syncthreads();
+    for (int u = warp; u < units; u += nwarps) {
+        const unsigned int m = sm.mask[u];
+        if ((m >> lane) & 1u) {
+            const long long k = k0 + u * 32 + lane;
+            const long long pos = (long long)sm.base + sm.off[u] + __popc(m & ((1u << lane) - 1u));
+            if (pos < p.capacity) p.out_idx[pos] = p.row_idx ? p.row_idx[k] : (int32_t)k;
+            else latch(p.ctl, AA_ERR_CAPACITY);
+        }
+    }
+}
+
+__device__ __forceinline__ bool next_tile(const ShrinkParams& p, TailSmem& sm, unsigned int& tile) {
+    __syncthreads();   // previous tile's readers of sm are done
+    if (threadIdx.x == 0) sm.tile = atomicAdd(&p.ctl->ticket, 1u);
+    __syncthreads();
+    tile = sm.tile;
+    return tile < p.n_tiles;
+}
+
+// Last CTA out re-arms the ticket counter and starts a new flag generation, so the next
+// scan on this context (a later launch on the same stream) needs no clearing pass.
+__device__ __forceinline__ void scan_epilogue(const ShrinkParams& p, unsigned int epoch) {
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const unsigned int prev = atomicAdd(&p.ctl->done, 1u);
+        if (prev == gridDim.x - 1) {
+            p.ctl->ticket = 0;
+            p.ctl->done = 0;
+            unsigned int e = (epoch + 1u) & 0x3FFFFFFFu;
+            p.ctl->epoch = e ? e : 1u;
+        }
+    }
+}
+
+__device__ __forceinline__ unsigned int read_epoch(const ShrinkParams& p) {
+    return *(volatile unsigned int*)&p.ctl->epoch;
+}
+
+// Row of candidate k, or -1 (latching AA_ERR_BAD_INDEX) when the candidate list points outside the store.
+__device__ __forceinline__ long long candidate_row(const ShrinkParams& p, long long k) {
+    if (!p.row_idx) return k;
+    const long long r = p.row_idx[k];
+    if ((unsigned long long)r >= (unsigned long long)p.n_stored) {
+        latch(p.ctl, AA_ERR_BAD_INDEX);
+        return -1;
+    }
+    return r;
+}
+
+// ---------------------------------------------------------------- dense linear Assistant
+// LPR lanes cooperate on one row; VEC = rows are 16-byte aligned and d is a whole number of vectors.
+template <typename T, int LPR, bool VEC>
+__global__ void __launch_bounds__(kScanThreads) score_shrink_dense_kernel(DenseFeat f, ShrinkParams p, int w_in_smem) {
+    extern __shared__ float w_smem[];
+    __shared__ TailSmem sm;
+    constexpr int VE = Vec<T>::kElems;
+    const int tid = threadIdx.x;
+    const float* wv = f.w;
+    if (w_in_smem) {
+        for (int j = tid; j < f.d; j += kScanThreads) w_smem[j] = f.w[j];
+        wv = w_smem;
+    }
+    const float bias = *f.b;
+    const unsigned int epoch = read_epoch(p);
+    const T* base = static_cast<const T*>(f.base);
+    constexpr int G = kScanThreads / LPR;
+    const int group = tid / LPR, gl = tid % LPR;
+    const int nvec = (int)(f.d / VE);
+
+    unsigned int tile;
+    while (next_tile(p, sm, tile)) {
+        const long long k0 = (long long)tile * p.tile_rows;
+        for (int rl = group; rl < p.tile_rows; rl += G) {
+            const long long k = k0 + rl;
+            const long long r = k < p.n_cand ? candidate_row(p, k) : -1;
+            float acc = 0.0f;
+            if (r >= 0) {
+                const T* row = base + r * f.row_stride;
+                if (VEC) {
+#pragma unroll 4
+                    for (int v = gl; v < nvec; v += LPR) {
+                        float x[VE];
+                        Vec<T>::load(row + (long long)v * VE, x);
+                        const float* wp = wv + (long long)v * VE;
+#pragma unroll
+                        for (int e = 0; e < VE; ++e) acc = fmaf(x[e], wp[e], acc);
+                    }
+                } else {
+                    for (long long j = gl; j < f.d; j += LPR) acc = fmaf(Vec<T>::one(row + j), wv[j], acc);
+                }
+            }
+#pragma unroll
+            for (int o = LPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+            if (gl == 0) sm.s[rl] = r >= 0 ? acc + bias : __int_as_float(0x7FC00000);
+        }
+        __syncthreads();
+        shrink_compact_tile(p, tile, epoch, sm);
+    }
+    scan_epilogue(p, epoch);
+}
+
+// ---------------------------------------------------------------- CSR bag-of-words Assistant
+template <int LPR>
+__global__ void __launch_bounds__(kScanThreads) score_shrink_csr_kernel(CsrFeat f, ShrinkParams p) {
+    __shared__ TailSmem sm;
+    const int tid = threadIdx.x;
+    const float bias = *f.b;
+    const unsigned int epoch = read_epoch(p);
+    constexpr int G = kScanThreads / LPR;
+    const int group = tid / LPR, gl = tid % LPR;
+
+    unsigned int tile;
+    while (next_tile(p, sm, tile)) {
+        const long long k0 = (long long)tile * p.tile_rows;
+        for (int rl = group; rl < p.tile_rows; rl += G) {
+            const long long k = k0 + rl;
+            const long long r = k < p.n_cand ? candidate_row(p, k) : -1;
+            float acc = 0.0f;
+            if (r >= 0) {
+                const int e0 = __ldg(f.indptr + r), e1 = __ldg(f.indptr + r + 1);
+                for (int e = e0 + gl; e < e1; e += LPR) {
+                    const int c = __ldg(f.col + e);
+                    if ((unsigned int)c < (unsigned long long)f.d) acc = fmaf(__ldg(f.val + e), __ldg(f.w + c), acc);
+                    else latch(p.ctl, AA_ERR_BAD_INDEX);
+                }
+            }
+#pragma unroll
+            for (int o = LPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+            if (gl == 0) sm.s[rl] = r >= 0 ? acc + bias : __int_as_float(0x7FC00000);
+        }
+        __syncthreads();
+        shrink_compact_tile(p, tile, epoch, sm);
+    }
+    scan_epilogue(p, epoch);
+}
+
+// ---------------------------------------------------------------- precomputed pre-activations
+__global__ void __launch_bounds__(kScanThreads) shrink_from_scores_kernel(const float* __restrict__ score, ShrinkParams p) {
+    __shared__ TailSmem sm;
+    const unsigned int epoch = read_epoch(p);
+    unsigned int tile;
+    while (next_tile(p, sm, tile)) {
+        const long long k0 = (long long)tile * p.tile_rows;
+        for (int rl = threadIdx.x; rl < p.tile_rows; rl += kScanThreads) {
+            const long long k = k0 + rl;
+            sm.s[rl] = k < p.n_cand ? __ldg(score + k) : 0.0f;
+        }
+        __syncthreads();
+        shrink_compact_tile(p, tile, epoch, sm);
+    }
+    scan_epilogue(p, epoch);
+}
+
+int pow2_ceil(int64_t v) {
+    int p = 1;
+    while (p < v) p <<= 1;
+    return p;
+}
+
+// Rows per tile: about `target_bytes` of input per tile, a multiple of 32, and small enough
+// that the pool splits into at least two tiles per SM when it is large enough to.
+int choose_tile_rows(const aa_ctx_impl* c, int64_t n_cand, double bytes_per_row, double target_bytes) {
+    int64_t rows = (int64_t)(target_bytes / (bytes_per_row > 1.0 ? bytes_per_row : 1.0));
+    const int64_t spread = n_cand / (2 * (int64_t)c->sm_count);
+    if (rows > spread) rows = spread;
+    rows = (rows / 32) * 32;
+    if (rows < 32) rows = 32;
+    if (rows > kMaxTileRows) rows = kMaxTileRows;
+    return (int)rows;
+}
+
+aa_status finish_params(aa_ctx_impl* c, ShrinkParams& sp, int tile_rows) {
+    sp.tile_rows = tile_rows;
+    const int64_t n_tiles = (sp.n_cand + tile_rows - 1) / tile_rows;
+    if (n_tiles > c->max_tiles) return AA_ERR_WORKSPACE;
+    sp.n_tiles = (unsigned int)n_tiles;
+    sp.ctl = c->ctl;
+    sp.tile_state = c->tile_state;
+    // flag generations repeat after 2^30 scans: clear the flags long before that can matter
+    if (++c->scans_since_clear >= (1ull << 29)) {
+        c->scans_since_clear = 0;
+        if (cudaMemsetAsync(c->tile_state, 0, sizeof(unsigned long long) * c->max_tiles, c->stream) != cudaSuccess)
+            return AA_ERR_CUDA;
+    }
+    return AA_OK;
+}
+
+template <typename K>
+aa_status launch_scan(aa_ctx_impl* c, K kernel, size_t smem, const ShrinkParams& sp, void** args) {
+    if (smem > 48 * 1024) {
+        if (cudaFuncSetAttribute((const void*)kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return AA_ERR_CUDA;
+    }
+    int grid = resident_ctas(c, (const void*)kernel, kScanThreads, smem);
+    if (grid <= 0) return AA_ERR_CUDA;
+    if ((unsigned int)grid > sp.n_tiles) grid = (int)sp.n_tiles;
+    if (cudaLaunchKernel((const void*)kernel, dim3(grid), dim3(kScanThreads), args, smem, c->stream) != cudaSuccess)
+        return AA_ERR_CUDA;
+    ++c->launches;
+    return AA_OK;
+}
+
+template <typename T, bool VEC>
+aa_status dispatch_dense(aa_ctx_impl* c, DenseFeat& f, ShrinkParams& sp, int lpr, size_t smem, int w_in_smem) {
+    void* args[] = {&f, &sp, &w_in_smem};
+    switch (lpr) {
+        case 4: return launch_scan(c, score_shrink_dense_kernel<T, 4, VEC>, smem, sp, args);
+        case 8: return launch_scan(c, score_shrink_dense_kernel<T, 8, VEC>, smem, sp, args);
+        case 16: return launch_scan(c, score_shrink_dense_kernel<T, 16, VEC>, smem, sp, args);
+        default: return launch_scan(c, score_shrink_dense_kernel<T, 32, VEC>, smem, sp, args);
+    }
+}
+
+}  // namespace
+
+aa_status launch_score_shrink_dense(aa_ctx_impl* c, const DenseFeat& f_in, ShrinkParams sp) {
+    DenseFeat f = f_in;
+    const int es = f.dtype == AA_BF16 ? 2 : 4;
+    const int ve = 16 / es;
+    const bool vec = ((uintptr_t)f.base % 16 == 0) && ((f.row_stride * es) % 16 == 0) && (f.d % ve == 0);
+    const int64_t work_items = vec ? f.d / ve : f.d;
+    int lpr = pow2_ceil((work_items + 1) / 2);
+    lpr = lpr < 4 ? 4 : (lpr > 32 ? 32 : lpr);
+    aa_status st = finish_params(c, sp, choose_tile_rows(c, sp.n_cand, (double)f.d * es, 192.0 * 1024));
+    if (st != AA_OK) return st;
+    // w is staged in shared memory when it fits beside the tile state with room for several CTAs per SM
+    const int w_in_smem = f.d * sizeof(float) <= 96 * 1024 ? 1 : 0;
+    const size_t smem = w_in_smem ? (size_t)f.d * sizeof(float) : 0;
+    if (f.dtype == AA_BF16)
+        return vec ? dispatch_dense<uint16_t, true>(c, f, sp, lpr, smem, w_in_smem)
+                   : dispatch_dense<uint16_t, false>(c, f, sp, lpr, smem, w_in_smem);
+    return vec ? dispatch_dense<float, true>(c, f, sp, lpr, smem, w_in_smem)
+               : dispatch_dense<float, false>(c, f, sp, lpr, smem, w_in_smem);
+}
+
+aa_status launch_score_shrink_csr(aa_ctx_impl* c, const CsrFeat& f_in, ShrinkParams sp) {
+    CsrFeat f = f_in;
+    int lpr = pow2_ceil((int64_t)(f.mean_nnz / 4.0f + 0.5f));
+    lpr = lpr < 4 ? 4 : (lpr > 32 ? 32 : lpr);
+    aa_status st = finish_params(c, sp, choose_tile_rows(c, sp.n_cand, 8.0 * f.mean_nnz + 4.0, 64.0 * 1024));
+    if (st != AA_OK) return st;
+    void* args[] = {&f, &sp};
+    switch (lpr) {
+        case 4: return launch_scan(c, score_shrink_csr_kernel<4>, 0, sp, args);
+        case 8: return launch_scan(c, score_shrink_csr_kernel<8>, 0, sp, args);
+        case 16: return launch_scan(c, score_shrink_csr_kernel<16>, 0, sp, args);
+        default: return launch_scan(c, score_shrink_csr_kernel<32>, 0, sp, args);
+    }
+}
+
+aa_status launch_shrink_from_scores(aa_ctx_impl* c, const float* score, ShrinkParams sp) {
+    aa_status st = finish_params(c, sp, choose_tile_rows(c, sp.n_cand, 4.0, 4.0 * kMaxTileRows));
+    if (st != AA_OK) return st;
+    void* args[] = {&score, &sp};
+    return launch_scan(c, shrink_from_scores_kernel, 0, sp, args);
+}
+
+}  // namespace aa
