@@ -132,6 +132,12 @@ struct Vec<float> {
         unpack(__ldg(reinterpret_cast<const uint4*>(p)), out);
     }
     __device__ static __forceinline__ float one(const float* p) { return __ldg(p); }
+    // weights staged in shared memory: plain order, lane v reads one float4 (conflict-free)
+    __device__ static __forceinline__ int w_index(int j, int /*nvec*/) { return j; }
+    __device__ static __forceinline__ void load_w(const float* w_s, int /*nvec*/, int v, float (&out)[4]) {
+        const float4 a = reinterpret_cast<const float4*>(w_s)[v];
+        out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
+    }
 };
 template <>
 struct Vec<uint16_t> {   // bf16 bit patterns
@@ -146,6 +152,18 @@ struct Vec<uint16_t> {   // bf16 bit patterns
         unpack(__ldg(reinterpret_cast<const uint4*>(p)), out);
     }
     __device__ static __forceinline__ float one(const uint16_t* p) { return __uint_as_float((uint32_t)__ldg(p) << 16); }
+    // weights staged in shared memory: the 8 weights of vector v are split into two float4
+    // planes so that consecutive lanes read consecutive 16-byte words (conflict-free)
+    __device__ static __forceinline__ int w_index(int j, int nvec) {
+        const int v = j >> 3, e = j & 7;
+        return (e >> 2) * nvec * 4 + v * 4 + (e & 3);
+    }
+    __device__ static __forceinline__ void load_w(const float* w_s, int nvec, int v, float (&out)[8]) {
+        const float4 a = reinterpret_cast<const float4*>(w_s)[v];
+        const float4 b = reinterpret_cast<const float4*>(w_s)[nvec + v];
+        out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
+        out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
+    }
 };
 
 #endif  // __CUDACC__
@@ -169,6 +187,11 @@ struct CsrFeat {
 };
 
 aa_status launch_score_shrink_dense(aa_ctx_impl* c, const DenseFeat& f, ShrinkParams sp);
+// Bulk-copy (cp.async.bulk + mbarrier) variant for 16-byte aligned rows; AA_ERR_UNSUPPORTED when
+// the shape does not fit its shared-memory ring, in which case the caller uses the load-based kernel.
+aa_status launch_score_shrink_dense_tma(aa_ctx_impl* c, const DenseFeat& f, ShrinkParams sp);
+// Tile geometry + scan state of a shrink launch (sets tile_rows, n_tiles, ctl, tile_state).
+aa_status finish_shrink_params(aa_ctx_impl* c, ShrinkParams& sp, int tile_rows);
 aa_status launch_score_shrink_csr(aa_ctx_impl* c, const CsrFeat& f, ShrinkParams sp);
 aa_status launch_shrink_from_scores(aa_ctx_impl* c, const float* score, ShrinkParams sp);
 

@@ -1,15 +1,13 @@
 // Assistant score -> Bernoulli shrink -> ordered batch list, fused in one pass
 // (Algorithm 1, Assistant.sample_batch, evaluated for a whole candidate pool at once).
 //
-// Every kernel here is a persistent grid.  A CTA repeatedly takes the next tile of
-// candidates from a ticket counter, computes the tile's pre-activations, draws the
-// keep/skip decision per candidate (Philox keyed by seed, counter = (instance id,
-// step)), and appends the kept candidates to the batch list at the position given by a
-// decoupled look-back scan over the tiles, so that the list keeps candidate order.
-// Tiles are handed out in look-back order, so every tile a CTA waits on is owned by a
-// CTA that is already running; each wait is still bounded and gives up with a latched
-// AA_ERR_SCAN_TIMEOUT instead of spinning for ever.
-#include "aa_internal.cuh"
+// The kernels in this file read the features with ordinary 128-bit (or element-wise) loads:
+// any alignment, any stride, CSR rows, or precomputed pre-activations.  A CTA repeatedly takes
+// the next tile of candidates from the ticket counter, computes the tile's pre-activations
+// into shared memory, then draws the keep/skip decisions and appends the kept candidates
+// (scan_tail.cuh).  Aligned dense rows normally take the bulk-copy kernel of
+// score_shrink_tma.cu instead.
+#include "scan_tail.cuh"
 
 namespace aa {
 
@@ -23,58 +21,6 @@ struct TailSmem {
     unsigned int tile;
 };
 
-__device__ __forceinline__ unsigned long long pack_state(unsigned int flag, int value) {
-    return ((unsigned long long)flag << 32) | (unsigned int)value;
-}
-
-// Decoupled look-back (warp-collective, called by warp 0): publishes this tile's count and
-// returns the number kept in all earlier tiles.
-__device__ int lookback_exclusive(const ShrinkParams& p, unsigned int tile, unsigned int epoch, int total) {
-    const int lane = threadIdx.x & 31;
-    const unsigned int flag_agg = epoch * 4u + 1u, flag_inc = epoch * 4u + 2u;
-    unsigned long long* state = p.tile_state;
-    if (tile == 0) {
-        if (lane == 0) st_relaxed_u64(&state[0], pack_state(flag_inc, total));
-        return 0;
-    }
-    if (lane == 0) st_relaxed_u64(&state[tile], pack_state(flag_agg, total));
-    int excl = 0;
-    long long window_end = (long long)tile - 1;
-    bool gave_up = false;
-    while (!gave_up) {
-        const long long idx = window_end - lane;
-        unsigned int flag = flag_inc;   // lanes before tile 0 stand for "inclusive prefix 0"
-        int val = 0;
-        unsigned int polls = 0;
-        while (true) {
-            if (idx >= 0) {
-                const unsigned long long w = ld_relaxed_u64(&state[idx]);
-                flag = (unsigned int)(w >> 32);
-                val = (int)(unsigned int)w;
-            }
-            const unsigned int inc_m = __ballot_sync(0xFFFFFFFFu, flag == flag_inc);
-            const unsigned int agg_m = __ballot_sync(0xFFFFFFFFu, flag == flag_agg);
-            // only the tiles between this one and the nearest inclusive prefix have to be ready
-            const unsigned int need = inc_m ? ((1u << (__ffs(inc_m) - 1)) - 1u) : 0xFFFFFFFFu;
-            if (((inc_m | agg_m) & need) == need) break;
-            if (++polls > kSpinLimit) { gave_up = true; break; }
-            __nanosleep(polls < 64 ? 32 : 256);
-        }
-        if (gave_up) break;
-        const unsigned int inc_m = __ballot_sync(0xFFFFFFFFu, flag == flag_inc);
-        const int first = inc_m ? (__ffs(inc_m) - 1) : 31;
-        int contrib = lane <= first ? val : 0;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) contrib += __shfl_xor_sync(0xFFFFFFFFu, contrib, o);
-        excl += contrib;
-        if (inc_m) break;
-        window_end -= 32;
-    }
-    if (gave_up && lane == 0) latch(p.ctl, AA_ERR_SCAN_TIMEOUT);
-    if (lane == 0) st_relaxed_u64(&state[tile], pack_state(flag_inc, excl + total));
-    return excl;
-}
-
 // Shrink decision + ordered append for one tile whose pre-activations are in sm.s.
 // All threads of the CTA call this; contains CTA barriers.
 __device__ void shrink_compact_tile(const ShrinkParams& p, unsigned int tile, unsigned int epoch, TailSmem& sm) {
@@ -87,11 +33,7 @@ __device__ void shrink_compact_tile(const ShrinkParams& p, unsigned int tile, un
         bool keep = false;
         if (k < p.n_cand) {
             const float s = sm.s[u * 32 + lane];
-            const long long r = p.row_idx ? (long long)p.row_idx[k] : k;
-            // net acceptance probability of Algorithm 1: gamma + (1 - gamma) g
-            const float prob = fmaf(1.0f - p.mix, sigmoid_f32(s), p.mix);
-            const float c = philox_uniform(p, (uint64_t)(p.id_base + r));
-            keep = c < prob;   // false for the NaN that marks an unreadable row
+            keep = keep_decision(p, k, s);
             if (p.out_score) p.out_score[k] = s;
             if (p.out_mask) p.out_mask[k] = keep ? 1 : 0;
         }
@@ -135,47 +77,22 @@ __device__ __forceinline__ bool next_tile(const ShrinkParams& p, TailSmem& sm, u
     return tile < p.n_tiles;
 }
 
-// Last CTA out re-arms the ticket counter and starts a new flag generation, so the next
-// scan on this context (a later launch on the same stream) needs no clearing pass.
-__device__ __forceinline__ void scan_epilogue(const ShrinkParams& p, unsigned int epoch) {
-    if (threadIdx.x == 0) {
-        __threadfence();
-        const unsigned int prev = atomicAdd(&p.ctl->done, 1u);
-        if (prev == gridDim.x - 1) {
-            p.ctl->ticket = 0;
-            p.ctl->done = 0;
-            unsigned int e = (epoch + 1u) & 0x3FFFFFFFu;
-            p.ctl->epoch = e ? e : 1u;
-        }
-    }
-}
-
-__device__ __forceinline__ unsigned int read_epoch(const ShrinkParams& p) {
-    return *(volatile unsigned int*)&p.ctl->epoch;
-}
-
-// Row of candidate k, or -1 (latching AA_ERR_BAD_INDEX) when the candidate list points outside the store.
-__device__ __forceinline__ long long candidate_row(const ShrinkParams& p, long long k) {
-    if (!p.row_idx) return k;
-    const long long r = p.row_idx[k];
-    if ((unsigned long long)r >= (unsigned long long)p.n_stored) {
-        latch(p.ctl, AA_ERR_BAD_INDEX);
-        return -1;
-    }
-    return r;
-}
+constexpr float kNaN = __builtin_nanf("");
 
 // ---------------------------------------------------------------- dense linear Assistant
-// LPR lanes cooperate on one row; VEC = rows are 16-byte aligned and d is a whole number of vectors.
+// LPR lanes cooperate on one row.  VEC: rows are 16-byte aligned, d is a whole number of
+// vectors and w sits in shared memory in the conflict-free vector layout.
 template <typename T, int LPR, bool VEC>
 __global__ void __launch_bounds__(kScanThreads) score_shrink_dense_kernel(DenseFeat f, ShrinkParams p, int w_in_smem) {
-    extern __shared__ float w_smem[];
+    extern __shared__ __align__(16) float w_smem[];
     __shared__ TailSmem sm;
     constexpr int VE = Vec<T>::kElems;
     const int tid = threadIdx.x;
+    const int nvec = (int)(f.d / VE);
     const float* wv = f.w;
     if (w_in_smem) {
-        for (int j = tid; j < f.d; j += kScanThreads) w_smem[j] = f.w[j];
+        if (VEC) for (int j = tid; j < f.d; j += kScanThreads) w_smem[Vec<T>::w_index(j, nvec)] = f.w[j];
+        else for (int j = tid; j < f.d; j += kScanThreads) w_smem[j] = f.w[j];
         wv = w_smem;
     }
     const float bias = *f.b;
@@ -183,7 +100,6 @@ __global__ void __launch_bounds__(kScanThreads) score_shrink_dense_kernel(DenseF
     const T* base = static_cast<const T*>(f.base);
     constexpr int G = kScanThreads / LPR;
     const int group = tid / LPR, gl = tid % LPR;
-    const int nvec = (int)(f.d / VE);
 
     unsigned int tile;
     while (next_tile(p, sm, tile)) {
@@ -197,11 +113,11 @@ __global__ void __launch_bounds__(kScanThreads) score_shrink_dense_kernel(DenseF
                 if (VEC) {
 #pragma unroll 4
                     for (int v = gl; v < nvec; v += LPR) {
-                        float x[VE];
+                        float x[VE], wq[VE];
                         Vec<T>::load(row + (long long)v * VE, x);
-                        const float* wp = wv + (long long)v * VE;
+                        Vec<T>::load_w(w_smem, nvec, v, wq);
 #pragma unroll
-                        for (int e = 0; e < VE; ++e) acc = fmaf(x[e], wp[e], acc);
+                        for (int e = 0; e < VE; ++e) acc = fmaf(x[e], wq[e], acc);
                     }
                 } else {
                     for (long long j = gl; j < f.d; j += LPR) acc = fmaf(Vec<T>::one(row + j), wv[j], acc);
@@ -209,7 +125,7 @@ __global__ void __launch_bounds__(kScanThreads) score_shrink_dense_kernel(DenseF
             }
 #pragma unroll
             for (int o = LPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-            if (gl == 0) sm.s[rl] = r >= 0 ? acc + bias : __int_as_float(0x7FC00000);
+            if (gl == 0) sm.s[rl] = r >= 0 ? acc + bias : kNaN;
         }
         __syncthreads();
         shrink_compact_tile(p, tile, epoch, sm);
@@ -238,13 +154,13 @@ __global__ void __launch_bounds__(kScanThreads) score_shrink_csr_kernel(CsrFeat 
                 const int e0 = __ldg(f.indptr + r), e1 = __ldg(f.indptr + r + 1);
                 for (int e = e0 + gl; e < e1; e += LPR) {
                     const int c = __ldg(f.col + e);
-                    if ((unsigned int)c < (unsigned long long)f.d) acc = fmaf(__ldg(f.val + e), __ldg(f.w + c), acc);
+                    if ((unsigned long long)(unsigned int)c < (unsigned long long)f.d) acc = fmaf(__ldg(f.val + e), __ldg(f.w + c), acc);
                     else latch(p.ctl, AA_ERR_BAD_INDEX);
                 }
             }
 #pragma unroll
             for (int o = LPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-            if (gl == 0) sm.s[rl] = r >= 0 ? acc + bias : __int_as_float(0x7FC00000);
+            if (gl == 0) sm.s[rl] = r >= 0 ? acc + bias : kNaN;
         }
         __syncthreads();
         shrink_compact_tile(p, tile, epoch, sm);
@@ -287,22 +203,6 @@ int choose_tile_rows(const aa_ctx_impl* c, int64_t n_cand, double bytes_per_row,
     return (int)rows;
 }
 
-aa_status finish_params(aa_ctx_impl* c, ShrinkParams& sp, int tile_rows) {
-    sp.tile_rows = tile_rows;
-    const int64_t n_tiles = (sp.n_cand + tile_rows - 1) / tile_rows;
-    if (n_tiles > c->max_tiles) return AA_ERR_WORKSPACE;
-    sp.n_tiles = (unsigned int)n_tiles;
-    sp.ctl = c->ctl;
-    sp.tile_state = c->tile_state;
-    // flag generations repeat after 2^30 scans: clear the flags long before that can matter
-    if (++c->scans_since_clear >= (1ull << 29)) {
-        c->scans_since_clear = 0;
-        if (cudaMemsetAsync(c->tile_state, 0, sizeof(unsigned long long) * c->max_tiles, c->stream) != cudaSuccess)
-            return AA_ERR_CUDA;
-    }
-    return AA_OK;
-}
-
 template <typename K>
 aa_status launch_scan(aa_ctx_impl* c, K kernel, size_t smem, const ShrinkParams& sp, void** args) {
     if (smem > 48 * 1024) {
@@ -331,17 +231,38 @@ aa_status dispatch_dense(aa_ctx_impl* c, DenseFeat& f, ShrinkParams& sp, int lpr
 
 }  // namespace
 
+aa_status finish_shrink_params(aa_ctx_impl* c, ShrinkParams& sp, int tile_rows) {
+    sp.tile_rows = tile_rows;
+    const int64_t n_tiles = (sp.n_cand + tile_rows - 1) / tile_rows;
+    if (n_tiles > c->max_tiles) return AA_ERR_WORKSPACE;
+    sp.n_tiles = (unsigned int)n_tiles;
+    sp.ctl = c->ctl;
+    sp.tile_state = c->tile_state;
+    // flag generations repeat after 2^30 scans: clear the flags long before that can matter
+    if (++c->scans_since_clear >= (1ull << 29)) {
+        c->scans_since_clear = 0;
+        if (cudaMemsetAsync(c->tile_state, 0, sizeof(unsigned long long) * c->max_tiles, c->stream) != cudaSuccess)
+            return AA_ERR_CUDA;
+    }
+    return AA_OK;
+}
+
 aa_status launch_score_shrink_dense(aa_ctx_impl* c, const DenseFeat& f_in, ShrinkParams sp) {
     DenseFeat f = f_in;
     const int es = f.dtype == AA_BF16 ? 2 : 4;
     const int ve = 16 / es;
-    const bool vec = ((uintptr_t)f.base % 16 == 0) && ((f.row_stride * es) % 16 == 0) && (f.d % ve == 0);
+    const bool aligned = ((uintptr_t)f.base % 16 == 0) && ((f.row_stride * es) % 16 == 0) && (f.d % ve == 0);
+    if (aligned) {
+        aa_status st = launch_score_shrink_dense_tma(c, f, sp);
+        if (st != AA_ERR_UNSUPPORTED) return st;
+    }
+    // the vector path keeps w in shared memory; otherwise rows are read element by element
+    const bool vec = aligned && f.d * sizeof(float) <= 96 * 1024;
     const int64_t work_items = vec ? f.d / ve : f.d;
     int lpr = pow2_ceil((work_items + 1) / 2);
     lpr = lpr < 4 ? 4 : (lpr > 32 ? 32 : lpr);
-    aa_status st = finish_params(c, sp, choose_tile_rows(c, sp.n_cand, (double)f.d * es, 192.0 * 1024));
+    aa_status st = finish_shrink_params(c, sp, choose_tile_rows(c, sp.n_cand, (double)f.d * es, 192.0 * 1024));
     if (st != AA_OK) return st;
-    // w is staged in shared memory when it fits beside the tile state with room for several CTAs per SM
     const int w_in_smem = f.d * sizeof(float) <= 96 * 1024 ? 1 : 0;
     const size_t smem = w_in_smem ? (size_t)f.d * sizeof(float) : 0;
     if (f.dtype == AA_BF16)
@@ -355,7 +276,7 @@ aa_status launch_score_shrink_csr(aa_ctx_impl* c, const CsrFeat& f_in, ShrinkPar
     CsrFeat f = f_in;
     int lpr = pow2_ceil((int64_t)(f.mean_nnz / 4.0f + 0.5f));
     lpr = lpr < 4 ? 4 : (lpr > 32 ? 32 : lpr);
-    aa_status st = finish_params(c, sp, choose_tile_rows(c, sp.n_cand, 8.0 * f.mean_nnz + 4.0, 64.0 * 1024));
+    aa_status st = finish_shrink_params(c, sp, choose_tile_rows(c, sp.n_cand, 8.0 * f.mean_nnz + 4.0, 64.0 * 1024));
     if (st != AA_OK) return st;
     void* args[] = {&f, &sp};
     switch (lpr) {
@@ -367,7 +288,7 @@ aa_status launch_score_shrink_csr(aa_ctx_impl* c, const CsrFeat& f_in, ShrinkPar
 }
 
 aa_status launch_shrink_from_scores(aa_ctx_impl* c, const float* score, ShrinkParams sp) {
-    aa_status st = finish_params(c, sp, choose_tile_rows(c, sp.n_cand, 4.0, 4.0 * kMaxTileRows));
+    aa_status st = finish_shrink_params(c, sp, choose_tile_rows(c, sp.n_cand, 4.0, 4.0 * kMaxTileRows));
     if (st != AA_OK) return st;
     void* args[] = {&score, &sp};
     return launch_scan(c, shrink_from_scores_kernel, 0, sp, args);
