@@ -10,70 +10,11 @@
 // onto the touched weights with fp32 atomics.
 #include <math.h>
 
-#include "aa_internal.cuh"
+#include "step_common.cuh"
 
 namespace aa {
 
 namespace {
-
-constexpr int kStepThreads = 512;
-constexpr int kStepWarps = kStepThreads / 32;
-
-struct StepParams {
-    DenseFeat f;
-    CsrFeat csr;
-    const int32_t* row_idx;
-    int64_t n_stored;
-    int64_t m_host;
-    const int32_t* count_dev;
-    const float* loss;
-    int thresh_mode;
-    float threshold;
-    float lr;
-    float* w;
-    float* b;
-    float* partials;      // [parts][d_pad] column sums, then [parts] bias sums
-    float* residual;      // per batch row (CSR path)
-    int64_t d_pad;
-    int rows_per_block;
-    Control* ctl;
-};
-
-__device__ __forceinline__ int64_t batch_size(const StepParams& p) {
-    int64_t m = p.m_host;
-    if (p.count_dev) {
-        const int64_t c = *p.count_dev;
-        m = c < 0 ? 0 : (c < m ? c : m);
-    }
-    return m;
-}
-
-// Shrinking threshold T: the caller's value, or the mean of the batch losses.  Every CTA adds the
-// losses in the same order (fp64), so all CTAs agree on T bit for bit.
-__device__ double block_threshold(const StepParams& p, int64_t m, double* red /* [warps] */) {
-    if (p.thresh_mode == AA_THRESH_VALUE) return (double)p.threshold;
-    double acc = 0.0;
-    for (int64_t i = threadIdx.x; i < m; i += blockDim.x) acc += (double)__ldg(p.loss + i);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-    if (lane == 0) red[warp] = acc;
-    __syncthreads();
-    double total = 0.0;
-    for (int wi = 0; wi < nwarps; ++wi) total += red[wi];
-    __syncthreads();
-    return m > 0 ? total / (double)m : 0.0;
-}
-
-__device__ __forceinline__ long long batch_row(const StepParams& p, int64_t i) {
-    if (!p.row_idx) return i;
-    const long long r = p.row_idx[i];
-    if ((unsigned long long)r >= (unsigned long long)p.n_stored) {
-        latch(p.ctl, AA_ERR_BAD_INDEX);
-        return -1;
-    }
-    return r;
-}
 
 // ---------------------------------------------------------------- dense
 // CI = 16-byte column vectors owned by each thread.  VEC = rows are 16-byte aligned.
@@ -197,21 +138,36 @@ __global__ void __launch_bounds__(kStepThreads) linear_grad_dense_kernel(StepPar
     }
 }
 
-// Adds the partials in CTA order and applies the SGD update.
+// Adds the partials and applies the SGD update.  A CTA owns 32 columns; its 8 warps each add a
+// strided share of the partials (loads in flight, not a serial chain) and the 8 shares are then
+// combined in a fixed order, so the result is reproducible for a given set of partials.
 __global__ void __launch_bounds__(256) linear_apply_kernel(StepParams p, int parts) {
+    __shared__ float share[8][33];
     const int64_t m = batch_size(p);
     if (m <= 0) return;
     const float scale = p.lr / (float)m;
-    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
+    const int64_t j = (int64_t)blockIdx.x * 32 + lane;
+    float g = 0.0f;
     if (j < p.f.d) {
-        float g = 0.0f;
-        for (int q = 0; q < parts; ++q) g += p.partials[(int64_t)q * p.d_pad + j];
-        p.w[j] = p.w[j] - scale * g;
+#pragma unroll 4
+        for (int q = grp; q < parts; q += 8) g += p.partials[(int64_t)q * p.d_pad + j];
     }
-    if (j == 0) {
-        float g = 0.0f;
-        for (int q = 0; q < parts; ++q) g += p.partials[(int64_t)parts * p.d_pad + q];
-        p.b[0] = p.b[0] - scale * g;
+    share[grp][lane] = g;
+    __syncthreads();
+    if (grp == 0 && j < p.f.d) {
+        float t = 0.0f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) t += share[k][lane];
+        p.w[j] = p.w[j] - scale * t;
+    }
+    if (blockIdx.x == 0 && grp == 1) {
+        // bias: the per-CTA residual sums sit behind the column partials
+        float t = 0.0f;
+        for (int q = lane; q < parts; q += 32) t += p.partials[(int64_t)parts * p.d_pad + q];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
+        if (lane == 0) p.b[0] = p.b[0] - scale * t;
     }
 }
 
@@ -291,6 +247,16 @@ const void* pick_dense_kernel(int ci) {
 
 }  // namespace
 
+aa_status launch_linear_apply(aa_ctx_impl* c, const StepParams& p_in, int parts) {
+    StepParams p = p_in;
+    void* args[] = {&p, &parts};
+    const int agrid = (int)((p.f.d + 31) / 32);
+    if (cudaLaunchKernel((const void*)linear_apply_kernel, dim3(agrid), dim3(256), args, 0, c->stream) != cudaSuccess)
+        return AA_ERR_CUDA;
+    ++c->launches;
+    return AA_OK;
+}
+
 aa_status launch_assistant_step_dense(aa_ctx_impl* c, const DenseFeat& f, const int32_t* row_idx, int64_t n_stored,
                                       int64_t m_host, const int32_t* count_dev, const float* loss, float* w, float* b,
                                       float lr, int thresh_mode, float threshold) {
@@ -313,6 +279,12 @@ aa_status launch_assistant_step_dense(aa_ctx_impl* c, const DenseFeat& f, const 
     p.partials = c->partials;
     p.ctl = c->ctl;
     p.d_pad = (f.d + ve - 1) / ve * ve;
+    if (vec) {
+        int parts = 0;
+        aa_status st = launch_assistant_grad_dense_tma(c, p, &parts);
+        if (st == AA_OK) return launch_linear_apply(c, p, parts);
+        if (st != AA_ERR_UNSUPPORTED) return st;
+    }
     const int64_t nvec = p.d_pad / ve;
     int ci = 1;
     while (ci < 8 && (int64_t)ci * kStepThreads < nvec) ci <<= 1;
@@ -343,13 +315,7 @@ aa_status launch_assistant_step_dense(aa_ctx_impl* c, const DenseFeat& f, const 
     void* args[] = {&p};
     if (cudaLaunchKernel(kernel, dim3(grid), dim3(kStepThreads), args, smem, c->stream) != cudaSuccess) return AA_ERR_CUDA;
     ++c->launches;
-    int parts = grid;
-    void* args2[] = {&p, &parts};
-    const int agrid = (int)((f.d + 255) / 256);
-    if (cudaLaunchKernel((const void*)linear_apply_kernel, dim3(agrid), dim3(256), args2, 0, c->stream) != cudaSuccess)
-        return AA_ERR_CUDA;
-    ++c->launches;
-    return AA_OK;
+    return launch_linear_apply(c, p, grid);
 }
 
 aa_status launch_assistant_step_csr(aa_ctx_impl* c, const CsrFeat& f, const int32_t* row_idx, int64_t n_stored,

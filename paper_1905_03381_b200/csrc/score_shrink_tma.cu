@@ -27,7 +27,7 @@ namespace aa {
 namespace {
 
 constexpr int kMaxRowBytes = 24 * 1024;              // longest row the ring takes
-constexpr int kTargetStage = 24 * 1024;              // preferred bytes of one ring stage
+constexpr int kTargetStage = 32 * 1024;              // preferred bytes of one ring stage
 constexpr int kMaxStages = 8;
 constexpr int kMaxSplit = 2;                         // consumer warps per stage
 constexpr int kConsumers = kMaxStages * kMaxSplit;
@@ -175,11 +175,16 @@ __global__ void __launch_bounds__(kTmaThreads, 1) score_shrink_tma_kernel(DenseF
         cb->abort_flag = 0;
         mbar_fence_init();
     }
-    for (int j = tid; j < f.d; j += kTmaThreads) w_s[Vec<T>::w_index(j, g.nvec)] = f.w[j];
     const float bias = *f.b;
     const unsigned int epoch = read_epoch(p);
     volatile int* abort_flag = &cb->abort_flag;
-    __syncthreads();
+    __syncthreads();   // barriers are initialised
+    // The consumer warps stage the weights among themselves (named barrier 1) while the
+    // producer is already streaming rows.
+    if (warp >= 1 && warp <= kConsumers) {
+        for (int j = tid - 32; j < f.d; j += kConsumers * 32) w_s[Vec<T>::w_index(j, g.nvec)] = f.w[j];
+        asm volatile("bar.sync 1, %0;" ::"n"(kConsumers * 32) : "memory");
+    }
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
