@@ -41,6 +41,8 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--cpu-steps", type=int, default=4, help="oracle steps timed for cpu_baseline (0 = skip)")
     ap.add_argument("--pool-rows", type=int, default=None, help="override the pool size (testing only)")
+    ap.add_argument("--loss-reps", type=int, default=20,
+                    help="timed calls of the per-sentence loss on the translation shape (0 = skip)")
     return ap.parse_args()
 
 
@@ -53,13 +55,34 @@ def measured_peak_gbs():
         return 6650.0, "fallback"
 
 
-def ncu_traffic_bytes():
-    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if still valid."""
-    path = os.path.join(ROOT, "profiles", "traffic.json")
+TRAFFIC_PROFILE = os.path.join(ROOT, "profiles", "score_shrink_tma_bf16_d3072.txt")
+TRAFFIC_SOURCES = ("score_shrink_tma.cu", "scan_tail.cuh", "async_copy.cuh", "aa_internal.cuh")
+
+
+def kernel_source_digest():
+    """SHA-256 over the sources of the dominant kernel, as recorded beside its ncu counters."""
+    import hashlib
+
+    h = hashlib.sha256()
+    for name in TRAFFIC_SOURCES:
+        with open(os.path.join(ROOT, "paper_1905_03381_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def ncu_traffic_bytes(candidates: int):
+    """DRAM bytes per launch of the dominant kernel, scaled from the committed ncu summary by the candidates
+    one launch screens; None when the summary is missing or the kernel's sources changed since the capture."""
     try:
-        with open(path) as f:
-            rec = json.load(f)
-        return rec.get("score_shrink_dense_bf16_n65536_d3072_dram_bytes_per_launch")
+        rec = {}
+        with open(TRAFFIC_PROFILE) as f:
+            for line in f:
+                if ":" in line and not line.startswith("#"):
+                    k, v = line.split(":", 1)
+                    rec[k.strip()] = v.strip()
+        if rec.get("source_sha256") != kernel_source_digest():
+            return None
+        return float(rec["dram_bytes_per_candidate"]) * candidates
     except Exception:
         return None
 
@@ -216,7 +239,10 @@ def run_b200(args, cfg):
     aa = B.AutoAssist(max_rows=cfg.n, max_d=cfg.d, device=dev)
     asst = B.linear_assistant(w, b)
     out_idx = torch.zeros(cfg.n, dtype=torch.int32, device=dev)
-    out_count = torch.zeros(1, dtype=torch.int32, device=dev)
+    # one device count per step, so that the mean batch size of the timed steps is known without a host read
+    n_slots = max(args.warmup, 3) + args.steps
+    counts = torch.zeros(n_slots, dtype=torch.int32, device=dev)
+    count_of = [counts[j:j + 1] for j in range(n_slots)]
     loss = torch.zeros(cfg.n, dtype=torch.float32, device=dev)
     feats = [B.dense_features(p, id_base=base) for p, base in zip(pools, plan.id_bases)]
     batch_feats = [B.dense_features(p, row_idx=out_idx, id_base=base) for p, base in zip(pools, plan.id_bases)]
@@ -225,6 +251,7 @@ def run_b200(args, cfg):
 
     def step(i, events=None):
         k = i % npool
+        out_count = count_of[i % n_slots]
         if events is not None:
             events[0].record()
         aa.aa_score_shrink(feats[k], asst, cfg.gamma, cfg.philox_seed, i, out_idx, out_count)
@@ -255,7 +282,6 @@ def run_b200(args, cfg):
         sampler.start()
         time.sleep(0.3)
     launches0 = aa.aa_launch_count()
-    accepted = 0
     barrier()
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_start.record()
@@ -270,12 +296,49 @@ def run_b200(args, cfg):
         sampler.stop()
     status = aa.aa_device_status()
     assert status == B.AA_OK, B.status_string(status)
-    accepted = int(out_count.item())
+    timed = counts[[(args.warmup + i) % n_slots for i in range(K)]].cpu().numpy().astype(np.int64)
+    accepted = float(timed.mean())            # mean batch size M over the timed steps
     score_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / K
     loss_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / K
     asst_ms = sum(e[2].elapsed_time(e[3]) for e in ev) / K
 
     agg = sharding.aggregate(dist if world > 1 else None, dev, elapsed_ms, cfg.n * K)
+
+    # ---- second half of the metric: per-instance-loss rows/s on the translation shape
+    # (25,000 token rows x 32,000-word bf16 logits = 1.6 GB per call, larger than L2; per-sentence sums)
+    loss_rows = None
+    if args.loss_reps > 0 and rank == 0:
+        t2 = W.TranslationShape()
+        rows2 = t2.token_budget
+        lg2 = t2.token_logits(rows2, dev)
+        ids2 = t2.token_ids(rows2, dev)
+        off2 = torch.from_numpy(W.ragged_offsets(rows2, t2.len_lo, t2.len_hi, 9)).to(dev)
+        sent_loss = torch.zeros(off2.numel() - 1, dtype=torch.float32, device=dev)
+        aa2 = B.AutoAssist(max_rows=rows2, max_d=8, device=dev)
+        g2 = B.logits_desc(lg2)
+        for _ in range(3):
+            aa2.aa_instance_loss(g2, ids2, sent_loss, offsets=off2)
+        torch.cuda.synchronize()
+        l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n0 = aa2.aa_launch_count()
+        l0.record()
+        for _ in range(args.loss_reps):
+            aa2.aa_instance_loss(g2, ids2, sent_loss, offsets=off2)
+        l1.record()
+        torch.cuda.synchronize()
+        assert aa2.aa_device_status() == B.AA_OK
+        ms2 = l0.elapsed_time(l1) / args.loss_reps
+        bytes2 = rows2 * t2.vocab * 2 + rows2 * 8 + off2.numel() * 4 + sent_loss.numel() * 4
+        peak2, kind2 = measured_peak_gbs()
+        loss_rows = {"workload": f"translation shape: {rows2} token rows x {t2.vocab} bf16 logits N(0,4), "
+                                 f"{sent_loss.numel()} sentences of 8..128 tokens, summed per sentence",
+                     "value": rows2 / (ms2 * 1e-3), "unit": "token rows/s", "ms_per_call": ms2,
+                     "launches_per_call": (aa2.aa_launch_count() - n0) // args.loss_reps,
+                     "roofline": {"bound": "hbm", "achieved": bytes2 / (ms2 * 1e-3) / 1e9, "peak": peak2, "unit": "GB/s",
+                                  "frac": bytes2 / (ms2 * 1e-3) / 1e9 / peak2, "peak_kind": f"of {kind2}",
+                                  "algorithmic_bytes_per_launch": bytes2}}
+        aa2.close()
+        del lg2, ids2, aa2
 
     # ---- end to end through the host-buffer entry point (pinned host inputs, results read back)
     e2e = None
@@ -316,7 +379,7 @@ def run_b200(args, cfg):
     alg_bytes = cfg.n * cfg.d * 2 + cfg.d * 4 + accepted * 4 + 4
     achieved = alg_bytes / (score_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "score_shrink_dense_kernel<bf16>", "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": ncu_traffic_bytes(),
+                "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": ncu_traffic_bytes(cfg.n),
                 "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": score_ms,
                 "frac_of_nominal_8TBs": achieved / 8000.0}
     loss_bytes = accepted * (cfg.classes * 4 + 8)
@@ -341,8 +404,8 @@ def run_b200(args, cfg):
         "metric": METRIC, "value": agg["units"] / (agg["ms"] * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": max(args.warmup, 3), "ms_per_step": agg["ms"] / K, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(cfg, args),
-        "roofline": roofline, "stages": stages, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
-        "accepted_last_step": accepted, "clocks": sampler.summary(),
+        "roofline": roofline, "stages": stages, "instance_loss_rows": loss_rows, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
+        "accepted_mean": accepted, "accepted_min": int(timed.min()), "accepted_max": int(timed.max()), "clocks": sampler.summary(),
     }
     print(json.dumps(line), flush=True)
     if world > 1:
