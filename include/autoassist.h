@@ -164,6 +164,38 @@ aa_status aa_shrink_compact(aa_ctx* ctx, const float* score, int64_t n, int64_t 
                             int32_t* out_idx, int64_t capacity, int32_t* out_count, uint8_t* out_mask);
 
 /*
+ * aa_shrink_compact for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a deployment variant of the entry point above.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits — a plug-in or callback inside a
+ * host application that owns the whole memory pool, a real-time loop that must not enter the
+ * allocator, a process that starts after the device memory has been handed out.  Such a caller
+ * cannot provide the workspace that aa_create wants, so this variant takes no context: its scan
+ * state (a control block and one look-back word per 1024-candidate tile, 33 KB) is a fixed array
+ * inside the library, present on every device that loads the library for the life of the process.
+ * The call itself allocates and frees nothing on host or device.
+ *
+ *   - n may be at most AA_STATIC_MAX_CANDIDATES; a larger n returns AA_ERR_WORKSPACE and enqueues
+ *     nothing.  Split a larger pool into consecutive calls with id_base advanced by the rows done.
+ *   - Inputs and outputs are the caller's device buffers exactly as for aa_shrink_compact; results
+ *     are bit-identical to it for the same arguments.
+ *   - out_status (nullable, device int32): receives the condition latched by this call
+ *     (AA_OK, AA_ERR_CAPACITY, AA_ERR_SCAN_TIMEOUT), ordered on the stream like the other outputs.
+ *   - cuda_stream: the cudaStream_t to enqueue on (NULL = legacy default stream), on the CURRENT device.
+ *   - The first call on each device looks up the array's device address and the launch shape
+ *     (a few host-side CUDA queries); make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Each call clears the part it uses before its
+ *     kernel runs, so calls that follow each other on one stream are independent; calls that can
+ *     overlap on the GPU (different streams, different host threads without ordering) race on the
+ *     array and give wrong batches.  Serialise them.
+ */
+#define AA_STATIC_MAX_CANDIDATES (1 << 22)
+aa_status aa_shrink_compact_static(const float* score, int64_t n, int64_t id_base, float mix,
+                                   uint64_t seed, uint64_t step,
+                                   int32_t* out_idx, int64_t capacity, int32_t* out_count, uint8_t* out_mask,
+                                   int32_t* out_status, void* cuda_stream);
+
+/*
  * Step 4: per-instance Boss loss.  Row r: l_r = log sum_c exp(logit[r][c]) - logit[r][labels[r]]
  * (one pass, running maximum, fp32).  labels[r] < 0 marks padding (contributes 0); labels[r] >=
  * cols contributes 0 and latches AA_ERR_BAD_INDEX.

@@ -26,8 +26,9 @@ AA_THRESH_VALUE, AA_THRESH_BATCH_MEAN = 0, 1
 EXPORTS = (
     "aa_status_string", "aa_workspace_bytes", "aa_create", "aa_destroy", "aa_score_shrink",
     "aa_shrink_compact", "aa_instance_loss", "aa_assistant_step", "aa_step_host_staging_bytes", "aa_step_host",
-    "aa_device_status", "aa_launch_count",
+    "aa_device_status", "aa_launch_count", "aa_shrink_compact_static",
 )
+AA_STATIC_MAX_CANDIDATES = 1 << 22
 
 
 class aa_feat(Structure):
@@ -82,6 +83,8 @@ def lib() -> ctypes.CDLL:
                                       c_void_p, c_int64, c_void_p, c_void_p, c_void_p]
         L.aa_shrink_compact.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_float, c_uint64, c_uint64,
                                         c_void_p, c_int64, c_void_p, c_void_p]
+        L.aa_shrink_compact_static.argtypes = [c_void_p, c_int64, c_int64, c_float, c_uint64, c_uint64,
+                                               c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_void_p]
         L.aa_instance_loss.argtypes = [c_void_p, POINTER(aa_logits), c_void_p, c_void_p, c_int64, c_void_p, c_void_p]
         L.aa_assistant_step.argtypes = [c_void_p, POINTER(aa_feat), c_void_p, c_void_p, POINTER(aa_assistant),
                                         c_float, c_int32, c_float]
@@ -98,6 +101,21 @@ def lib() -> ctypes.CDLL:
 
 def status_string(status: int) -> str:
     return lib().aa_status_string(status).decode()
+
+
+def aa_shrink_compact_static(score: torch.Tensor, mix: float, seed: int, step: int, out_idx: torch.Tensor,
+                             out_count: torch.Tensor, out_mask=None, out_status=None, id_base: int = 0, n=None,
+                             stream=None):
+    """Shrink + compact on precomputed scores with no context and no workspace: the scan state is a fixed
+    array inside the library (for callers that cannot allocate device memory).  At most
+    AA_STATIC_MAX_CANDIDATES scores per call; calls on one device must not overlap."""
+    with torch.cuda.device(score.device):
+        s = stream if stream is not None else torch.cuda.current_stream(score.device)
+        st = lib().aa_shrink_compact_static(score.data_ptr(), score.numel() if n is None else n, id_base, mix, seed,
+                                            step, out_idx.data_ptr(), out_idx.numel(), out_count.data_ptr(),
+                                            _ptr(out_mask), _ptr(out_status), s.cuda_stream)
+    if st != AA_OK:
+        raise AutoAssistError(st, "aa_shrink_compact_static")
 
 
 def _ptr(t):

@@ -7,6 +7,10 @@
 // into shared memory, then draws the keep/skip decisions and appends the kept candidates
 // (scan_tail.cuh).  Aligned dense rows normally take the bulk-copy kernel of
 // score_shrink_tma.cu instead.
+#include <string.h>
+
+#include <mutex>
+
 #include "scan_tail.cuh"
 
 namespace aa {
@@ -295,3 +299,107 @@ aa_status launch_shrink_from_scores(aa_ctx_impl* c, const float* score, ShrinkPa
 }
 
 }  // namespace aa
+
+// ---------------------------------------------------------------- shrink + compact without any allocation
+// The scan state of this variant (control block + one look-back word per 1024-candidate tile)
+// lives in a file-scope device array instead of a caller-provided workspace.  Every device that
+// loads the library holds the array until the process exits.
+namespace aa {
+namespace {
+
+constexpr int64_t kStaticMaxCandidates = AA_STATIC_MAX_CANDIDATES;
+constexpr int kStaticTileRows = kMaxTileRows;
+constexpr int64_t kStaticMaxTiles = kStaticMaxCandidates / kStaticTileRows;
+static_assert(kStaticMaxCandidates % kStaticTileRows == 0, "whole tiles");
+
+struct StaticScan {
+    Control ctl;
+    unsigned long long tile_state[kStaticMaxTiles];
+};
+
+static __device__ __align__(256) unsigned char g_static_scan[sizeof(StaticScan)];
+
+// Host-side record per device: the array's device address (the symbol itself is only a host
+// stand-in) and the kernel's resident-CTA count.
+struct StaticScanDevice {
+    bool ready;
+    StaticScan* scan;
+    int grid_cap;
+};
+constexpr int kStaticMaxDevices = 64;
+StaticScanDevice g_static_dev[kStaticMaxDevices];
+std::mutex g_static_mutex;
+
+aa_status static_scan_for_current_device(StaticScanDevice& out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return AA_ERR_CUDA;
+    if (dev < 0 || dev >= kStaticMaxDevices) return AA_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticScanDevice& d = g_static_dev[dev];
+    if (!d.ready) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scan) != cudaSuccess || !ptr) return AA_ERR_CUDA;
+        int sms = 0, per_sm = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, (const void*)shrink_from_scores_kernel, kScanThreads, 0) != cudaSuccess ||
+            per_sm < 1)
+            return AA_ERR_CUDA;
+        d.scan = static_cast<StaticScan*>(ptr);
+        d.grid_cap = per_sm * sms;
+        d.ready = true;
+    }
+    out = d;
+    return AA_OK;
+}
+
+}  // namespace
+}  // namespace aa
+
+extern "C" aa_status aa_shrink_compact_static(const float* score, int64_t n, int64_t id_base, float mix, uint64_t seed,
+                                              uint64_t step, int32_t* out_idx, int64_t capacity, int32_t* out_count,
+                                              uint8_t* out_mask, int32_t* out_status, void* cuda_stream) {
+    using namespace aa;
+    if (!out_count || capacity < 0 || (capacity > 0 && !out_idx) || !(mix >= 0.0f && mix <= 1.0f)) return AA_ERR_INVALID_ARG;
+    if (n < 0 || (n > 0 && !score)) return AA_ERR_INVALID_ARG;
+    if (n > kStaticMaxCandidates) return AA_ERR_WORKSPACE;   // beyond what the built-in scratch array covers
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    StaticScanDevice dev;
+    aa_status st = static_scan_for_current_device(dev);
+    if (st != AA_OK) return st;
+    if (n == 0) {
+        if (cudaMemsetAsync(out_count, 0, sizeof(int32_t), stream) != cudaSuccess) return AA_ERR_CUDA;
+        if (out_status && cudaMemsetAsync(out_status, 0, sizeof(int32_t), stream) != cudaSuccess) return AA_ERR_CUDA;
+        return AA_OK;
+    }
+    ShrinkParams sp;
+    memset(&sp, 0, sizeof sp);
+    sp.n_cand = n;
+    sp.n_stored = n;
+    sp.id_base = id_base;
+    sp.mix = mix;
+    sp.seed_lo = (uint32_t)seed;
+    sp.seed_hi = (uint32_t)(seed >> 32);
+    sp.step_lo = (uint32_t)step;
+    sp.step_hi = (uint32_t)(step >> 32);
+    sp.out_idx = out_idx;
+    sp.capacity = capacity;
+    sp.out_count = out_count;
+    sp.out_mask = out_mask;
+    sp.tile_rows = kStaticTileRows;
+    sp.n_tiles = (unsigned int)((n + kStaticTileRows - 1) / kStaticTileRows);
+    sp.ctl = &dev.scan->ctl;
+    sp.tile_state = dev.scan->tile_state;
+    // The array keeps whatever the previous call left: ticket, counters, flag generation, status
+    // and this call's look-back words all start from zero.
+    const size_t used = sizeof(Control) + sizeof(unsigned long long) * sp.n_tiles;
+    if (cudaMemsetAsync(dev.scan, 0, used, stream) != cudaSuccess) return AA_ERR_CUDA;
+    int grid = dev.grid_cap;
+    if ((unsigned int)grid > sp.n_tiles) grid = (int)sp.n_tiles;
+    void* args[] = {&score, &sp};
+    if (cudaLaunchKernel((const void*)shrink_from_scores_kernel, dim3(grid), dim3(kScanThreads), args, 0, stream) != cudaSuccess)
+        return AA_ERR_CUDA;
+    if (out_status &&
+        cudaMemcpyAsync(out_status, &dev.scan->ctl.status, sizeof(int32_t), cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+        return AA_ERR_CUDA;
+    return AA_OK;
+}
