@@ -177,6 +177,20 @@ def linear_assistant(w: torch.Tensor, b: torch.Tensor) -> aa_assistant:
     return a
 
 
+def mlp_assistant(W1: torch.Tensor, W1_bf16: torch.Tensor, b1: torch.Tensor, w2: torch.Tensor, b2: torch.Tensor) -> aa_assistant:
+    """Two-layer Assistant: W1 fp32 master [hidden, d], its bf16 copy, b1[hidden], w2[hidden], b2[1]."""
+    for t, name in ((W1, "W1"), (b1, "b1"), (w2, "w2"), (b2, "b2")):
+        _check(t, torch.float32, name)
+    _check(W1_bf16, torch.bfloat16, "W1_bf16")
+    if W1.dim() != 2 or W1_bf16.shape != W1.shape or b1.numel() != W1.shape[0] or w2.numel() != W1.shape[0]:
+        raise TypeError("W1 must be [hidden, d] with matching W1_bf16, b1[hidden], w2[hidden]")
+    a = aa_assistant()
+    a.kind, a.hidden, a.d = AA_ASSIST_MLP, W1.shape[0], W1.shape[1]
+    a.W1, a.W1_bf16, a.b1, a.w2, a.b2 = W1.data_ptr(), W1_bf16.data_ptr(), b1.data_ptr(), w2.data_ptr(), b2.data_ptr()
+    a._keep = (W1, W1_bf16, b1, w2, b2)
+    return a
+
+
 def logits_desc(logits: torch.Tensor, rows=None) -> aa_logits:
     if logits.dim() != 2 or logits.stride(1) != 1 or not logits.is_cuda:
         raise TypeError("logits must be a 2-D CUDA tensor with contiguous rows")

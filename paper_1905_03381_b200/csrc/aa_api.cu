@@ -204,7 +204,15 @@ aa_status aa_score_shrink(aa_ctx* ctx, const aa_feat* feat, const aa_assistant* 
                             out_count, out_score, out_mask);
     if (st != AA_OK) return st;
     if (n_cand > c->max_rows || feat->d > c->max_d) return AA_ERR_WORKSPACE;
-    if (a->kind != AA_ASSIST_LINEAR) return AA_ERR_UNSUPPORTED;
+    if (a->kind == AA_ASSIST_MLP) {
+        if (a->d != feat->d || a->hidden <= 0 || !a->W1_bf16 || !a->b1 || !a->w2 || !a->b2) return AA_ERR_INVALID_ARG;
+        if (a->hidden > c->max_hidden) return AA_ERR_WORKSPACE;
+        if (feat->kind != AA_FEAT_DENSE || feat->dtype != AA_BF16) return AA_ERR_UNSUPPORTED;
+        if (n_cand == 0) return cuda_ok(cudaMemsetAsync(out_count, 0, sizeof(int32_t), c->stream));
+        MlpFeat f = {feat->dense, feat->n, feat->d, feat->row_stride, a->W1_bf16, a->b1, a->w2, a->b2, a->hidden};
+        return launch_score_shrink_mlp(c, f, sp);
+    }
+    if (a->kind != AA_ASSIST_LINEAR) return AA_ERR_INVALID_ARG;
     if (a->d != feat->d || !a->w || !a->b) return AA_ERR_INVALID_ARG;
     if (n_cand == 0) return cuda_ok(cudaMemsetAsync(out_count, 0, sizeof(int32_t), c->stream));
     if (feat->kind == AA_FEAT_DENSE) {

@@ -186,6 +186,19 @@ struct CsrFeat {
     float mean_nnz;
 };
 
+// Two-layer Assistant on dense bf16 rows: W1_bf16 is [hidden x d] row-major.
+struct MlpFeat {
+    const void* x;
+    int64_t n, d, row_stride;
+    const void* W1_bf16;
+    const float* b1;
+    const float* w2;
+    const float* b2;
+    int64_t hidden;
+};
+// tcgen05 scoring kernel (aligned bf16 rows, hidden a multiple of 16 up to 256, no candidate list).
+aa_status launch_score_shrink_mlp(aa_ctx_impl* c, const MlpFeat& f, ShrinkParams sp);
+
 aa_status launch_score_shrink_dense(aa_ctx_impl* c, const DenseFeat& f, ShrinkParams sp);
 // Bulk-copy (cp.async.bulk + mbarrier) variant for 16-byte aligned rows; AA_ERR_UNSUPPORTED when
 // the shape does not fit its shared-memory ring, in which case the caller uses the load-based kernel.

@@ -1,0 +1,147 @@
+"""Parity of the two-layer (tensor-core) Assistant with the CPU oracle.
+
+Bars: pre-activation scores |s - s_ref| <= 1e-5 (|s_ref| + sum_j |w2_j| ||W1_j|| ||x_i||), i.e. relative to the
+scale of the terms the two layers add up (bf16 products are exact in fp32; only the accumulation order differs);
+keep/skip mask bit-exact outside the tie band |p - c| < 1e-5; batch list bit-exact given the mask.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import aa_oracle as O
+from paper_1905_03381_b200 import binding as B
+from paper_1905_03381_b200 import build, workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def aa():
+    build.build()
+    ctx = B.AutoAssist(max_rows=1 << 19, max_d=4096, max_hidden=256, device=DEV)
+    yield ctx
+    torch.cuda.synchronize()
+    assert ctx.aa_device_status() == B.AA_OK
+    ctx.close()
+
+
+def bf16_values(t):
+    """fp64 NumPy array of the values a bf16 tensor holds."""
+    return t.float().double().cpu().numpy()
+
+
+def make_mlp(d, hidden, seed, b1_std=0.2, b2=0.1):
+    W1, b1, w2, _ = W.mlp_assistant(d, hidden, seed, DEV)
+    b1 = W.normal((hidden,), b1_std, seed + 5, torch.float32, DEV)
+    b2_t = torch.full((1,), b2, dtype=torch.float32, device=DEV)
+    W1b = W1.to(torch.bfloat16).contiguous()
+    return W1, W1b, b1, w2, b2_t
+
+
+def mlp_screen(aa, x, params, mix, seed, step, id_base=0):
+    W1, W1b, b1, w2, b2 = params
+    n = x.shape[0]
+    out_idx = torch.full((n,), -7, dtype=torch.int32, device=DEV)
+    out_count = torch.full((1,), -7, dtype=torch.int32, device=DEV)
+    out_score = torch.zeros(n, dtype=torch.float32, device=DEV)
+    out_mask = torch.full((n,), 9, dtype=torch.uint8, device=DEV)
+    aa.aa_score_shrink(B.dense_features(x, id_base=id_base), B.mlp_assistant(W1, W1b, b1, w2, b2), mix, seed, step,
+                       out_idx, out_count, out_score, out_mask)
+    torch.cuda.synchronize()
+    return out_idx.cpu().numpy(), int(out_count.item()), out_score.cpu().numpy(), out_mask.cpu().numpy()
+
+
+def check_against_oracle(gpu, x_rows, params, mix, seed, step, ids):
+    """x_rows: the bf16 rows (tensor) the oracle scores; ids: their instance ids."""
+    idx, m, s, mask = gpu
+    W1, W1b, b1, w2, b2 = params
+    W1v = bf16_values(W1b)
+    s_ref = O.score_mlp(W.to_oracle(x_rows.contiguous()), W1v, b1.cpu().numpy(), w2.cpu().numpy(), float(b2.item()))
+    xn = np.linalg.norm(bf16_values(x_rows), axis=1)
+    scale = float(np.sum(np.abs(w2.double().cpu().numpy()) * np.linalg.norm(W1v, axis=1))) * xn
+    tol = 1e-5 * (np.abs(s_ref) + scale)
+    assert np.all(np.abs(s - s_ref) <= tol), float(np.max(np.abs(s - s_ref) / tol))
+    g = O.sigmoid(s_ref)
+    p = O.accept_prob(g, mix)
+    c = O.uniform(seed, step, ids)
+    keep = O.shrink(g, mix, seed, step, row_idx=np.asarray(ids, np.int32))
+    far = np.abs(p - c) >= 1e-5
+    return s_ref, keep, far
+
+
+@pytest.mark.parametrize("n,d,hidden", [
+    (1, 64, 16), (255, 64, 64), (257, 192, 32), (1000, 200, 64), (777, 3072, 256), (2048, 1000, 256), (5000, 128, 240),
+])
+def test_mlp_screen_matches_the_oracle(aa, n, d, hidden):
+    x = W.normal((n, d), 1.0, 90 + n, torch.bfloat16, DEV)
+    params = make_mlp(d, hidden, 91 + d)
+    mix, seed, step = 0.1, 7, n
+    gpu = mlp_screen(aa, x, params, mix, seed, step)
+    idx, m, s, mask = gpu
+    ids = np.arange(n)
+    s_ref, keep, far = check_against_oracle(gpu, x, params, mix, seed, step, ids)
+    assert set(np.unique(mask)) <= {0, 1}
+    assert np.array_equal(mask[far], keep[far])
+    assert m == int(mask.sum()) and np.array_equal(idx[:m], O.compact(mask))
+    assert np.all(idx[m:] == -7)
+    assert np.std(s_ref) > 0.05 or n == 1      # the case exercises a non-trivial score range
+
+
+def test_mlp_reduces_to_known_forms_on_the_gpu(aa):
+    # selector W1 (unit rows), w2 = 1, zero biases: s_i = sum_j relu(x_ij) over the first `hidden` features
+    n, d, hidden = 600, 128, 64
+    x = W.normal((n, d), 1.0, 5, torch.bfloat16, DEV)
+    W1 = torch.zeros((hidden, d), device=DEV)
+    W1[torch.arange(hidden), torch.arange(hidden)] = 1.0
+    params = (W1, W1.to(torch.bfloat16), torch.zeros(hidden, device=DEV), torch.ones(hidden, device=DEV), torch.zeros(1, device=DEV))
+    _, _, s, _ = mlp_screen(aa, x, params, 0.1, 1, 1)
+    expect = torch.relu(x[:, :hidden].float()).double().sum(1).cpu().numpy()
+    assert np.max(np.abs(s - expect)) <= 1e-5 * (np.abs(expect).max() + 1)
+
+
+def test_mlp_strided_rows_offset_ids_and_repeatability(aa):
+    n, d, hidden = 3000, 256, 128
+    buf = W.normal((n, d + 8), 1.0, 6, torch.bfloat16, DEV)
+    x = buf[:, :d]                                   # row stride d + 8 elements (16-byte aligned)
+    params = make_mlp(d, hidden, 17)
+    base = (1 << 32) - 77
+    gpu = mlp_screen(aa, x, params, 0.3, (1 << 40) + 1, 12, id_base=base)
+    idx, m, s, mask = gpu
+    W1, W1b, b1, w2, b2 = params
+    s_ref = O.score_mlp(W.to_oracle(x.contiguous()), bf16_values(W1b), b1.cpu().numpy(), w2.cpu().numpy(), float(b2.item()))
+    g = O.sigmoid(s_ref)
+    keep = O.shrink(g, 0.3, (1 << 40) + 1, 12, id_base=base)
+    c = O.uniform((1 << 40) + 1, 12, np.arange(n) + base)
+    far = np.abs(O.accept_prob(g, 0.3) - c) >= 1e-5
+    assert np.array_equal(mask[far], keep[far])
+    assert m == int(mask.sum()) and np.array_equal(idx[:m], O.compact(mask))
+    again = mlp_screen(aa, x, params, 0.3, (1 << 40) + 1, 12, id_base=base)
+    assert again[1] == m and np.array_equal(again[0], idx) and np.array_equal(again[2], s)
+
+
+def test_mlp_full_size_pool_sampled(aa):
+    """The MLP shape at full size (262,144 x 3072, hidden 256) in the launch configuration that is timed."""
+    cfg = W.MlpShape()
+    x = cfg.pool(DEV)
+    W1, b1, w2, b2 = cfg.assistant(DEV)
+    params = (W1, W1.to(torch.bfloat16).contiguous(), b1, w2, b2)
+    idx, m, s, mask = mlp_screen(aa, x, params, cfg.gamma, cfg.philox_seed, 3)
+    assert m == int(mask.sum()) and np.array_equal(idx[:m], np.nonzero(mask)[0])
+    sample = np.unique(np.concatenate([np.arange(40), np.arange(cfg.n - 40, cfg.n),
+                                       np.random.default_rng(4).integers(0, cfg.n, 300)])).astype(np.int64)
+    xs = x[torch.from_numpy(sample).to(DEV)]
+    W1v = bf16_values(params[1])
+    s_ref = O.score_mlp(W.to_oracle(xs.contiguous()), W1v, b1.cpu().numpy(), w2.cpu().numpy(), 0.0)
+    xn = np.linalg.norm(bf16_values(xs), axis=1)
+    scale = float(np.sum(np.abs(w2.double().cpu().numpy()) * np.linalg.norm(W1v, axis=1))) * xn
+    assert np.all(np.abs(s[sample] - s_ref) <= 1e-5 * (np.abs(s_ref) + scale))
+    g = O.sigmoid(s_ref)
+    c = O.uniform(cfg.philox_seed, 3, sample)
+    keep = O.shrink(g, cfg.gamma, cfg.philox_seed, 3, row_idx=sample.astype(np.int32))
+    far = np.abs(O.accept_prob(g, cfg.gamma) - c) >= 1e-5
+    assert np.array_equal(mask[sample][far], keep[far])
+    p_all = O.accept_prob(O.sigmoid(s.astype(np.float64)), cfg.gamma)
+    assert abs(m - p_all.sum()) < 5 * math.sqrt((p_all * (1 - p_all)).sum())
