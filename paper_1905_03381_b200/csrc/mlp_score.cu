@@ -7,8 +7,9 @@
 // One persistent CTA per SM, 12 warps.  A CTA owns super-tiles of 256 candidates: two 128-row
 // accumulators [128 x hidden] fp32 side by side in tensor memory, so that every 64-wide K-slice
 // of W1 fetched into shared memory is used for 256 candidates.
-//   warp 0      : TMA producer.  Per K-slice one box of 256 feature rows x 64 columns and one
-//                 box of `hidden` W1 rows x 64 columns (128-byte swizzle) into a 3-stage ring.
+//   warp 0      : TMA producer.  Per K-slice 256 feature rows x 64 columns (one box, or 64
+//                 four-row gathers when a candidate list selects the rows) and one box of
+//                 `hidden` W1 rows x 64 columns (128-byte swizzle) into a 3-stage ring.
 //   warp 1      : issues tcgen05.mma (M = 128, N = hidden, K = 16; 8 per stage), commits each
 //                 stage back to the producer and the finished super-tile to the epilogue.
 //   warp 2      : owns the TMEM allocation; then the tail: Philox keep/skip decisions of
@@ -19,161 +20,81 @@
 // Super-tiles are assigned round-robin (tile = blockIdx.x + k * gridDim.x); the grid never
 // exceeds the SM count, so every tile a look-back waits on belongs to a resident CTA.  All
 // waits are bounded and give up with AA_ERR_SCAN_TIMEOUT latched.
+#include "mlp_pipeline.cuh"
 #include "scan_tail.cuh"
-#include "tensor_core.cuh"
 
 namespace aa {
 
 namespace {
 
 constexpr int kMlpThreads = 384;
-constexpr int kSuperRows = 256;                 // candidates per super-tile (two M = 128 accumulators)
-constexpr int kSliceK = 64;                     // bf16 elements per 128-byte swizzled row
-constexpr int kMlpStages = 3;
-constexpr int kABytes = kSuperRows * 128;       // feature slice of one stage
-constexpr int kMaxHidden = 256;
 constexpr int kEpiWarps = 8;
-constexpr int kTmemCols = 512;
 
-struct MlpControl {
-    uint64_t full[kMlpStages], empty[kMlpStages];
-    uint64_t acc_full, acc_empty, drain;
+struct ScoreControl {
+    TilePipe pipe;
     uint64_t s_full[2], s_empty[2];
-    uint32_t tmem_base;
-    int abort_flag;
 };
 
 struct MlpKernelParams {
     const float* b1;
     const float* w2;
     const float* b2;
-    int hidden;
-    int k_slices;          // ceil(d / 64)
-    uint32_t b_bytes;      // hidden * 128
-    uint32_t stage_bytes;  // kABytes + b_bytes rounded up to 1024
+    MlpGeom g;
 };
 
-__device__ __forceinline__ void mlp_give_up(const ShrinkParams& p, MlpControl* cb) {
+__device__ __forceinline__ void mlp_give_up(const ShrinkParams& p, TilePipe* tp) {
     latch(p.ctl, AA_ERR_SCAN_TIMEOUT);
-    *(volatile int*)&cb->abort_flag = 1;
+    *(volatile int*)&tp->abort_flag = 1;
 }
 
+template <bool GATHER>
 __global__ void __launch_bounds__(kMlpThreads, 1)
 mlp_score_shrink_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                         MlpKernelParams mp, ShrinkParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* ring = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    float* b1_s = reinterpret_cast<float*>(ring + (size_t)kMlpStages * mp.stage_bytes);
+    float* b1_s = reinterpret_cast<float*>(ring + (size_t)kMlpStages * mp.g.stage_bytes);
     float* w2_s = b1_s + kMaxHidden;
     float* s_tile = w2_s + kMaxHidden;                      // [2][kSuperRows]
-    MlpControl* cb = reinterpret_cast<MlpControl*>(s_tile + 2 * kSuperRows);
+    ScoreControl* cb = reinterpret_cast<ScoreControl*>(s_tile + 2 * kSuperRows);
+    TilePipe* tp = &cb->pipe;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
-        for (int s = 0; s < kMlpStages; ++s) {
-            mbar_init(&cb->full[s], 1);
-            mbar_init(&cb->empty[s], 1);
-        }
-        mbar_init(&cb->acc_full, 1);
-        mbar_init(&cb->acc_empty, kEpiWarps);
-        mbar_init(&cb->drain, 1);
+        tile_pipe_init(tp, kEpiWarps);
         for (int q = 0; q < 2; ++q) {
             mbar_init(&cb->s_full[q], kEpiWarps);
             mbar_init(&cb->s_empty[q], 1);
         }
-        cb->abort_flag = 0;
         mbar_fence_init();
         prefetch_tensormap(&map_x);
         prefetch_tensormap(&map_w);
     }
     for (int j = tid; j < kMaxHidden; j += kMlpThreads) {
-        b1_s[j] = j < mp.hidden ? mp.b1[j] : 0.0f;
-        w2_s[j] = j < mp.hidden ? mp.w2[j] : 0.0f;
+        b1_s[j] = j < mp.g.hidden ? mp.b1[j] : 0.0f;
+        w2_s[j] = j < mp.g.hidden ? mp.w2[j] : 0.0f;
     }
-    if (warp == 2) tmem_alloc(&cb->tmem_base, kTmemCols);
+    if (warp == 2) tmem_alloc(&tp->tmem_base, kTmemCols);
     const unsigned int epoch = read_epoch(p);
-    volatile int* abort_flag = &cb->abort_flag;
+    volatile int* abort_flag = &tp->abort_flag;
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    const uint32_t tmem_base = *(volatile uint32_t*)&cb->tmem_base;
+    const uint32_t tmem_base = *(volatile uint32_t*)&tp->tmem_base;
     const unsigned int n_tiles = p.n_tiles;
 
     if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
-        int stage = 0, j = 0;
-        uint32_t phase = 0;
-        bool ok = true;
-        for (unsigned int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-            const int row0 = (int)(tile * (unsigned int)kSuperRows);
-            for (int ks = 0; ks < mp.k_slices; ++ks) {
-                if (!mbar_wait(&cb->empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
-                if (lane == 0) {
-                    unsigned char* a_dst = ring + (size_t)stage * mp.stage_bytes;
-                    mbar_arrive_expect_tx(&cb->full[stage], (uint32_t)kABytes + mp.b_bytes);
-                    tma_load_2d(a_dst, &map_x, ks * kSliceK, row0, &cb->full[stage]);
-                    tma_load_2d(a_dst + kABytes, &map_w, ks * kSliceK, 0, &cb->full[stage]);
-                }
-                __syncwarp();
-                ++j;
-                if (++stage == kMlpStages) { stage = 0; phase ^= 1u; }
-            }
-        }
-        if (!ok) {
-            if (lane == 0) mlp_give_up(p, cb);
-            // let copies still in flight land before the CTA's shared memory goes away
-            const int pending = j < kMlpStages ? j : kMlpStages;
-            for (int back = 1; back <= pending; ++back) {
-                const int jj = j - back, st = jj % kMlpStages, use = jj / kMlpStages;
-                const long long t0 = clock64();
-                while (!mbar_try_wait(&cb->full[st], (uint32_t)(use & 1)) && clock64() - t0 < kWaitCycles) {}
-            }
-        }
+        if (!mlp_produce<GATHER>(tp, ring, &map_x, &map_w, mp.g, n_tiles, p.row_idx, p.n_cand, p.n_stored) && lane == 0)
+            mlp_give_up(p, tp);
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        const uint32_t idesc = umma_idesc_bf16(128, mp.hidden, false, false);
-        int stage = 0, it = 0;
-        uint32_t phase = 0;
-        bool ok = true;
-        for (unsigned int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
-            // the epilogue has drained both accumulators of the previous super-tile
-            if (!mbar_wait(&cb->acc_empty, (uint32_t)((it & 1) ^ 1), abort_flag)) { ok = false; break; }
-            tc_fence_after_sync();
-            for (int ks = 0; ks < mp.k_slices; ++ks) {
-                if (!mbar_wait(&cb->full[stage], phase, abort_flag)) { ok = false; break; }
-                tc_fence_after_sync();
-                if (lane == 0) {
-                    const uint32_t a_addr = smem_u32(ring + (size_t)stage * mp.stage_bytes);
-                    const uint32_t b_addr = a_addr + kABytes;
-#pragma unroll
-                    for (int k = 0; k < kSliceK / 16; ++k) {
-                        const uint64_t b_desc = umma_smem_desc(b_addr + k * 32, 16, 1024);
-                        const bool acc = (ks | k) != 0;
-                        umma_bf16(tmem_base, umma_smem_desc(a_addr + k * 32, 16, 1024), b_desc, idesc, acc);
-                        umma_bf16(tmem_base + kMaxHidden, umma_smem_desc(a_addr + 128 * 128 + k * 32, 16, 1024), b_desc, idesc, acc);
-                    }
-                    umma_commit(&cb->empty[stage]);                               // stage reusable once these MMAs are done
-                    if (ks == mp.k_slices - 1) umma_commit(&cb->acc_full);        // super-tile finished
-                }
-                __syncwarp();
-                if (++stage == kMlpStages) { stage = 0; phase ^= 1u; }
-            }
-        }
-        if (!ok && lane == 0) mlp_give_up(p, cb);
-        // every MMA issued by this thread has retired before the tensor memory is released
-        if (lane == 0) umma_commit(&cb->drain);
-        __syncwarp();
-        {
-            const long long t0 = clock64();
-            while (!mbar_try_wait(&cb->drain, 0) && clock64() - t0 < kWaitCycles) {}
-        }
+        if (!mlp_issue_mma(tp, ring, mp.g, n_tiles, tmem_base) && lane == 0) mlp_give_up(p, tp);
     } else if (warp == 2) {
         // ------------------------------------------------------------ tail: shrink + ordered append
         int it = 0;
         for (unsigned int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
             const int buf = it & 1;
             if (!mbar_wait(&cb->s_full[buf], (uint32_t)((it >> 1) & 1), abort_flag)) {
-                if (lane == 0) mlp_give_up(p, cb);
+                if (lane == 0) mlp_give_up(p, tp);
                 break;
             }
             float sv[kSuperRows / 32];
@@ -181,6 +102,14 @@ mlp_score_shrink_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
             for (int u = 0; u < kSuperRows / 32; ++u) sv[u] = s_tile[buf * kSuperRows + u * 32 + lane];
             __syncwarp();
             if (lane == 0) mbar_arrive(&cb->s_empty[buf]);
+            if (GATHER) {
+                // a list entry outside the stored rows was scored on a stand-in row: void it (and latch)
+#pragma unroll
+                for (int u = 0; u < kSuperRows / 32; ++u) {
+                    const long long k = (long long)tile * kSuperRows + u * 32 + lane;
+                    if (k < p.n_cand && candidate_row(p, k) < 0) sv[u] = __builtin_nanf("");
+                }
+            }
             warp_shrink_compact<kSuperRows / 32>(p, tile, epoch, kSuperRows / 32, sv);
         }
     } else if (warp >= 4) {
@@ -193,14 +122,14 @@ mlp_score_shrink_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
         int it = 0;
         for (unsigned int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
             const int buf = it & 1;
-            if (!mbar_wait(&cb->acc_full, (uint32_t)(it & 1), abort_flag) ||
+            if (!mbar_wait(&tp->acc_full, (uint32_t)(it & 1), abort_flag) ||
                 !mbar_wait(&cb->s_empty[buf], (uint32_t)(((it >> 1) & 1) ^ 1), abort_flag)) {
-                if (lane == 0) mlp_give_up(p, cb);
+                if (lane == 0) mlp_give_up(p, tp);
                 break;
             }
             tc_fence_after_sync();
             float s = 0.0f;
-            for (int c0 = 0; c0 < mp.hidden; c0 += 32) {
+            for (int c0 = 0; c0 < mp.g.hidden; c0 += 32) {
                 uint32_t r[32];
                 tmem_ld_32cols(t_row + (uint32_t)c0, r);
                 tmem_ld_wait();
@@ -218,7 +147,7 @@ mlp_score_shrink_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(&cb->acc_empty);
+                mbar_arrive(&tp->acc_empty);
                 mbar_arrive(&cb->s_full[buf]);
             }
         }
@@ -257,25 +186,22 @@ bool encode_bf16_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uin
 
 aa_status launch_score_shrink_mlp(aa_ctx_impl* c, const MlpFeat& f, ShrinkParams sp) {
     if (f.hidden < 16 || f.hidden > kMaxHidden || f.hidden % 16) return AA_ERR_UNSUPPORTED;
-    if (sp.row_idx) return AA_ERR_UNSUPPORTED;   // candidates are the stored rows in order
     if ((uintptr_t)f.x % 16 || (f.row_stride * 2) % 16 || (uintptr_t)f.W1_bf16 % 16 || (f.d * 2) % 16) return AA_ERR_UNSUPPORTED;
+    const bool gather = sp.row_idx != nullptr;
     alignas(64) CUtensorMap map_x, map_w;
-    if (!encode_bf16_tile_map(&map_x, f.x, (uint64_t)f.n, (uint64_t)f.d, (uint64_t)f.row_stride, kSuperRows) ||
+    if (!encode_bf16_tile_map(&map_x, f.x, (uint64_t)f.n, (uint64_t)f.d, (uint64_t)f.row_stride, gather ? 1 : kSuperRows) ||
         !encode_bf16_tile_map(&map_w, f.W1_bf16, (uint64_t)f.hidden, (uint64_t)f.d, (uint64_t)f.d, (uint32_t)f.hidden))
         return AA_ERR_CUDA;
     MlpKernelParams mp;
     mp.b1 = f.b1;
     mp.w2 = f.w2;
     mp.b2 = f.b2;
-    mp.hidden = (int)f.hidden;
-    mp.k_slices = (int)((f.d + kSliceK - 1) / kSliceK);
-    mp.b_bytes = (uint32_t)f.hidden * 128u;
-    mp.stage_bytes = ((uint32_t)kABytes + mp.b_bytes + 1023u) & ~1023u;
+    mp.g = make_mlp_geom(f.d, f.hidden);
     aa_status st = finish_shrink_params(c, sp, kSuperRows);
     if (st != AA_OK) return st;
-    const size_t smem = 1024 + (size_t)kMlpStages * mp.stage_bytes + sizeof(float) * (2 * kMaxHidden + 2 * kSuperRows) +
-                        sizeof(MlpControl) + 64;
-    const void* kernel = (const void*)mlp_score_shrink_kernel;
+    const size_t smem = 1024 + (size_t)kMlpStages * mp.g.stage_bytes + sizeof(float) * (2 * kMaxHidden + 2 * kSuperRows) +
+                        sizeof(ScoreControl) + 64;
+    const void* kernel = gather ? (const void*)mlp_score_shrink_kernel<true> : (const void*)mlp_score_shrink_kernel<false>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return AA_ERR_CUDA;
     int grid = c->sm_count;
     if ((unsigned int)grid > sp.n_tiles) grid = (int)sp.n_tiles;

@@ -122,6 +122,42 @@ def test_mlp_strided_rows_offset_ids_and_repeatability(aa):
     assert again[1] == m and np.array_equal(again[0], idx) and np.array_equal(again[2], s)
 
 
+def test_mlp_candidate_list_gathers_rows(aa):
+    n_store, n, d, hidden = 1500, 1000, 320, 96
+    x = W.normal((n_store, d), 1.0, 30, torch.bfloat16, DEV)
+    params = make_mlp(d, hidden, 31)
+    W1, W1b, b1, w2, b2 = params
+    rows = np.random.default_rng(32).permutation(n_store)[:n].astype(np.int32)
+    rows_t = torch.from_numpy(rows).to(DEV)
+    out_idx = torch.full((n,), -7, dtype=torch.int32, device=DEV)
+    out_count = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out_score = torch.zeros(n, dtype=torch.float32, device=DEV)
+    out_mask = torch.zeros(n, dtype=torch.uint8, device=DEV)
+    aa.aa_score_shrink(B.dense_features(x, row_idx=rows_t, id_base=10), B.mlp_assistant(W1, W1b, b1, w2, b2), 0.2, 3, 4,
+                       out_idx, out_count, out_score, out_mask)
+    torch.cuda.synchronize()
+    m, s, mask, idx = int(out_count.item()), out_score.cpu().numpy(), out_mask.cpu().numpy(), out_idx.cpu().numpy()
+    W1v = bf16_values(W1b)
+    s_ref = O.score_mlp(W.to_oracle(x), W1v, b1.cpu().numpy(), w2.cpu().numpy(), float(b2.item()), row_idx=rows)
+    xn = np.linalg.norm(bf16_values(x)[rows], axis=1)
+    scale = float(np.sum(np.abs(w2.double().cpu().numpy()) * np.linalg.norm(W1v, axis=1))) * xn
+    assert np.all(np.abs(s - s_ref) <= 1e-5 * (np.abs(s_ref) + scale))
+    g = O.sigmoid(s_ref)
+    keep = O.shrink(g, 0.2, 3, 4, id_base=10, row_idx=rows)
+    c = O.uniform(3, 4, rows.astype(np.int64) + 10)
+    far = np.abs(O.accept_prob(g, 0.2) - c) >= 1e-5
+    assert np.array_equal(mask[far], keep[far])
+    assert m == int(mask.sum()) and np.array_equal(idx[:m], O.compact(mask, row_idx=rows))
+    # an entry outside the stored rows is skipped and latched
+    bad = rows_t.clone(); bad[5] = n_store; bad[700] = -3
+    aa.aa_score_shrink(B.dense_features(x, row_idx=bad, id_base=10), B.mlp_assistant(W1, W1b, b1, w2, b2), 1.0, 3, 4,
+                       out_idx, out_count, out_score, out_mask)
+    torch.cuda.synchronize()
+    mask = out_mask.cpu().numpy()
+    assert mask[5] == 0 and mask[700] == 0 and int(out_count.item()) == n - 2
+    assert aa.aa_device_status() == B.AA_ERR_BAD_INDEX
+
+
 def test_mlp_full_size_pool_sampled(aa):
     """The MLP shape at full size (262,144 x 3072, hidden 256) in the launch configuration that is timed."""
     cfg = W.MlpShape()
