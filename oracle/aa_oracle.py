@@ -298,3 +298,23 @@ def assistant_step_linear_csr(indptr, col, val, f, w, b, lr, T=None, row_idx=Non
     w_new = sgd(w, gw, lr)
     b_new = sgd(np.array([b], np.float32), np.array([gb]), lr)[0]
     return w_new, b_new, z
+
+
+def assistant_step_mlp(x, f, W1, W1_bf16, b1, w2, b2, lr, T=None, row_idx=None):
+    """Two-layer Assistant: labels from losses f, back-propagation under the current parameters, one SGD update.
+
+    The forward pass reads the bf16 copy of W1 (uint16 bit patterns, as scoring does); the update goes to the fp32
+    master, which is then rounded to nearest even into the new bf16 copy.
+    Returns dict(W1, W1_bf16, b1, w2, b2, z, grads=(gW1, gb1, gw2, gb2), a, s).
+    """
+    f = _arr(f, np.float32)
+    W1_vals = (np.ascontiguousarray(W1_bf16, np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    T = batch_mean(f) if T is None else float(T)
+    z = labels(f, T)
+    s, a = score_mlp(x, W1_vals, b1, w2, b2, row_idx=row_idx, n_cand=f.size, want_pre=True)
+    gW1, gb1, gw2, gb2 = mlp_grad(x, a, s, z, w2, row_idx=row_idx)
+    W1_new = sgd(W1, gW1, lr)
+    return {
+        "W1": W1_new, "W1_bf16": round_bf16(W1_new), "b1": sgd(b1, gb1, lr), "w2": sgd(w2, gw2, lr),
+        "b2": sgd(np.array([b2], np.float32), np.array([gb2]), lr)[0], "z": z, "grads": (gW1, gb1, gw2, gb2), "a": a, "s": s,
+    }

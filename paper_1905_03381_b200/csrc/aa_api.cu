@@ -14,11 +14,11 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
     size_t tile_state_off, row_scratch_off, partials_off, total;
+    size_t mlp_pt_off, mlp_small_off, mlp_part_off, mlp_part_bytes;   // two-layer Assistant step (max_hidden > 0)
     int64_t max_tiles, partial_floats;
 };
 
 Layout make_layout(int64_t max_rows, int64_t max_d, int64_t max_hidden) {
-    (void)max_hidden;
     Layout L;
     L.max_tiles = (max_rows + 31) / 32 + 1;
     size_t off = sizeof(Control);
@@ -35,6 +35,14 @@ Layout make_layout(int64_t max_rows, int64_t max_d, int64_t max_hidden) {
     if (floats < 2 * d_pad) floats = 2 * d_pad;
     L.partial_floats = floats;
     off = align_up(off + sizeof(float) * (size_t)floats, 256);
+    L.mlp_pt_off = L.mlp_small_off = L.mlp_part_off = L.mlp_part_bytes = 0;
+    if (max_hidden > 0) {
+        size_t pt_bytes = 0, small_bytes = 0;
+        L.mlp_part_bytes = mlp_step_workspace_bytes(max_rows, max_d, max_hidden, &pt_bytes, &small_bytes);
+        L.mlp_pt_off = off;    off = align_up(off + pt_bytes, 1024);
+        L.mlp_small_off = off; off = align_up(off + small_bytes, 256);
+        L.mlp_part_off = off;  off = align_up(off + L.mlp_part_bytes, 256);
+    }
     L.total = off;
     return L;
 }
@@ -171,6 +179,12 @@ aa_status aa_create(aa_ctx** out, int64_t max_rows, int64_t max_d, int64_t max_h
     c.row_scratch = reinterpret_cast<float*>(c.ws + L.row_scratch_off);
     c.partials = reinterpret_cast<float*>(c.ws + L.partials_off);
     c.partial_floats = L.partial_floats;
+    if (max_hidden > 0) {
+        c.mlp_pt = c.ws + L.mlp_pt_off;
+        c.mlp_small = reinterpret_cast<float*>(c.ws + L.mlp_small_off);
+        c.mlp_part = reinterpret_cast<float*>(c.ws + L.mlp_part_off);
+        c.mlp_part_bytes = L.mlp_part_bytes;
+    }
     // control block and look-back flags start cleared; the flag generation starts at 1
     if (cudaMemsetAsync(c.ws, 0, L.row_scratch_off, c.stream) != cudaSuccess) {
         delete ctx;
@@ -259,7 +273,13 @@ aa_status aa_assistant_step(aa_ctx* ctx, const aa_feat* feat, const float* loss,
     aa_ctx_impl* c = &ctx->impl;
     const int64_t m_host = feat->row_idx ? feat->n_rows : feat->n;
     if (m_host > 0 && !loss) return AA_ERR_INVALID_ARG;
-    if (a->kind != AA_ASSIST_LINEAR) return AA_ERR_UNSUPPORTED;
+    if (a->kind == AA_ASSIST_MLP) {
+        if (a->d != feat->d || a->hidden <= 0 || !a->W1 || !a->W1_bf16 || !a->b1 || !a->w2 || !a->b2) return AA_ERR_INVALID_ARG;
+        if (feat->kind != AA_FEAT_DENSE || feat->dtype != AA_BF16) return AA_ERR_UNSUPPORTED;
+        MlpFeat f = {feat->dense, feat->n, feat->d, feat->row_stride, a->W1_bf16, a->b1, a->w2, a->b2, a->hidden};
+        return launch_assistant_step_mlp(c, f, a->W1, feat->row_idx, feat->n, m_host, count_dev, loss, lr, thresh_mode, threshold);
+    }
+    if (a->kind != AA_ASSIST_LINEAR) return AA_ERR_INVALID_ARG;
     if (a->d != feat->d || !a->w || !a->b) return AA_ERR_INVALID_ARG;
     if (feat->d > c->max_d) return AA_ERR_WORKSPACE;
     if (feat->kind == AA_FEAT_DENSE) {

@@ -39,6 +39,11 @@ struct aa_ctx_impl {
     int64_t partial_floats;
     int64_t launches;
     uint64_t scans_since_clear;
+    // two-layer Assistant step (present when the context was sized with max_hidden > 0)
+    void* mlp_pt;                     // bf16 [max_hidden][rows rounded up to 256]
+    float* mlp_small;                 // per-CTA column-sum partials
+    float* mlp_part;                  // split-K partials of the W1 gradient
+    size_t mlp_part_bytes;
 };
 
 // Arguments of the shrink + compaction tail shared by every scoring front end.
@@ -198,6 +203,13 @@ struct MlpFeat {
 };
 // tcgen05 scoring kernel (aligned bf16 rows, hidden a multiple of 16 up to 256, no candidate list).
 aa_status launch_score_shrink_mlp(aa_ctx_impl* c, const MlpFeat& f, ShrinkParams sp);
+
+// Labels + one SGD step of the two-layer Assistant on the batch rows (updates W1_master, W1_bf16, b1, w2, b2).
+aa_status launch_assistant_step_mlp(aa_ctx_impl* c, const MlpFeat& f, float* W1_master, const int32_t* row_idx, int64_t n_stored,
+                                    int64_t m_host, const int32_t* count_dev, const float* loss, float lr, int thresh_mode,
+                                    float threshold);
+// Workspace of that step: returns the bytes of the split-K partials, sets the bytes of P^T and of the column-sum partials.
+size_t mlp_step_workspace_bytes(int64_t max_rows, int64_t max_d, int64_t max_hidden, size_t* pt_bytes, size_t* small_bytes);
 
 aa_status launch_score_shrink_dense(aa_ctx_impl* c, const DenseFeat& f, ShrinkParams sp);
 // Bulk-copy (cp.async.bulk + mbarrier) variant for 16-byte aligned rows; AA_ERR_UNSUPPORTED when

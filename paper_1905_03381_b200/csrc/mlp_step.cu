@@ -1,0 +1,544 @@
+// Labels + one SGD step of the two-layer Assistant g = sigmoid(w2 . relu(W1 x + b1) + b2)
+// (Sec. 5.2 label rule and objective; Algorithm 2: Assistant.gradient, Assistant.update),
+// back-propagated through both layers on the tcgen05 tensor cores.
+//
+//   mlp_residual_kernel  forward pass over the batch rows under the current parameters (same
+//                        TMA/MMA pipeline as scoring), then per row  z = 1[loss > T],
+//                        r = sigmoid(s) - z,  and per hidden unit u the factor
+//                        P[i][u] = r_i [a_iu > 0]  of delta1_iu = r_i w2_u [a_iu > 0].
+//                        P is stored transposed in bf16 ([hidden x rows]); the column sums
+//                        sum_i r_i relu(a_iu) (-> grad w2), sum_i P[i][u] (-> grad b1) and
+//                        sum_i r_i (-> grad b2) stay in fp32 and leave as per-CTA partials.
+//   mlp_w1_grad_kernel   G[u][k] = sum_i P[i][u] x_ik : a [hidden x rows] x [rows x d] contraction
+//                        over the batch rows.  A CTA owns 256 feature columns and a slice of
+//                        the rows (split-K): per 64-row slice, P^T as a K-major operand and the
+//                        feature rows themselves as an MN-major operand (the contraction runs
+//                        down the rows, 128-byte swizzle), two [128 x 256] fp32 accumulators in
+//                        TMEM (hidden units 0..127 and 128..255).  Partials go to the workspace.
+//   mlp_apply_w1_kernel  W1 <- W1 - lr (w2_u / M) sum_splits G ; W1_bf16 <- round-to-nearest-even(W1).
+//   mlp_apply_small_kernel  b1, w2, b2 from the column-sum partials (reads the old w2 first).
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include "mlp_pipeline.cuh"
+#include "step_common.cuh"
+
+namespace aa {
+
+namespace {
+
+constexpr int kStepMlpThreads = 384;
+constexpr int kStepEpiWarps = 8;
+constexpr int kMaxMlpCtas = 192;              // bound on the grids below (workspace sizing)
+constexpr int kFeatChunk = 256;               // feature columns per CTA of the W1-gradient kernel
+constexpr int kRowSlice = 64;                 // batch rows per K-slice of the W1-gradient kernel
+
+struct MlpStepParams {
+    // batch
+    const int32_t* row_idx;
+    int64_t n_stored, m_host;
+    const int32_t* count_dev;
+    const float* loss;
+    int thresh_mode;
+    float threshold;
+    float lr;
+    // parameters
+    float* W1;
+    __nv_bfloat16* W1_bf16;
+    float* b1;
+    float* w2;
+    float* b2;
+    int64_t d;
+    MlpGeom g;
+    // workspace
+    __nv_bfloat16* Pt;        // [hidden][pitch]
+    int64_t pitch;
+    float* small;             // [ctas][2 * kMaxHidden + 1]: sum r relu(a), sum P, sum r
+    float* part;              // [splits][hidden][d_pad]
+    int64_t d_pad;
+    int n_chunks, splits;
+    Control* ctl;
+};
+
+__device__ __forceinline__ int64_t mlp_batch_size(const MlpStepParams& p) {
+    int64_t m = p.m_host;
+    if (p.count_dev) {
+        const int64_t c = *p.count_dev;
+        m = c < 0 ? 0 : (c < m ? c : m);
+    }
+    return m;
+}
+
+// Sum over the warp's 32 lanes of each of 32 per-lane values: afterwards v[0] of lane l holds the
+// total of element l (31 shuffles instead of 32 five-step reductions).
+__device__ __forceinline__ float lanes_transpose_sum(float (&v)[32], int lane) {
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+        const bool upper = (lane & off) != 0;
+#pragma unroll
+        for (int j = 0; j < off; ++j) {
+            const float send = upper ? v[j] : v[j + off];
+            const float keep = upper ? v[j + off] : v[j];
+            v[j] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, off);
+        }
+    }
+    return v[0];
+}
+
+__device__ __forceinline__ void step_give_up(const MlpStepParams& p, TilePipe* tp) {
+    latch(p.ctl, AA_ERR_SCAN_TIMEOUT);
+    *(volatile int*)&tp->abort_flag = 1;
+}
+
+// ---------------------------------------------------------------- forward + residuals + P^T
+template <bool GATHER>
+__global__ void __launch_bounds__(kStepMlpThreads, 1)
+mlp_residual_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, MlpStepParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* ring = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    float* b1_s = reinterpret_cast<float*>(ring + (size_t)kMlpStages * p.g.stage_bytes);
+    float* w2_s = b1_s + kMaxHidden;
+    float* col_s = w2_s + kMaxHidden;                        // [kStepEpiWarps][2][kMaxHidden] column sums per warp
+    double* red = reinterpret_cast<double*>(col_s + kStepEpiWarps * 2 * kMaxHidden);   // [warps]
+    float* rsum_s = reinterpret_cast<float*>(red + kStepMlpThreads / 32);              // [kStepEpiWarps]
+    TilePipe* tp = reinterpret_cast<TilePipe*>(rsum_s + kStepEpiWarps);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int hidden = p.g.hidden;
+    if (tid == 0) {
+        tile_pipe_init(tp, kStepEpiWarps);
+        mbar_fence_init();
+        prefetch_tensormap(&map_x);
+        prefetch_tensormap(&map_w);
+    }
+    for (int j = tid; j < kMaxHidden; j += kStepMlpThreads) {
+        b1_s[j] = j < hidden ? p.b1[j] : 0.0f;
+        w2_s[j] = j < hidden ? p.w2[j] : 0.0f;
+    }
+    if (warp == 2) tmem_alloc(&tp->tmem_base, kTmemCols);
+    const int64_t m = mlp_batch_size(p);
+    // shrinking threshold T: the caller's value or the batch mean; every CTA adds the losses in the same order
+    double T_shrink = (double)p.threshold;
+    if (p.thresh_mode != AA_THRESH_VALUE) {
+        double acc = 0.0;
+        for (int64_t i = tid; i < m; i += kStepMlpThreads) acc += (double)__ldg(p.loss + i);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+        if (lane == 0) red[warp] = acc;
+    }
+    volatile int* abort_flag = &tp->abort_flag;
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    if (p.thresh_mode != AA_THRESH_VALUE) {
+        double total = 0.0;
+        for (int wi = 0; wi < kStepMlpThreads / 32; ++wi) total += red[wi];
+        T_shrink = m > 0 ? total / (double)m : 0.0;
+    }
+    const uint32_t tmem_base = *(volatile uint32_t*)&tp->tmem_base;
+    const unsigned int n_tiles = (unsigned int)((m + kSuperRows - 1) / kSuperRows);
+
+    if (warp == 0) {
+        if (!mlp_produce<GATHER>(tp, ring, &map_x, &map_w, p.g, n_tiles, p.row_idx, m, p.n_stored) && lane == 0) step_give_up(p, tp);
+    } else if (warp == 1) {
+        if (!mlp_issue_mma(tp, ring, p.g, n_tiles, tmem_base) && lane == 0) step_give_up(p, tp);
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------ epilogue
+        const int ew = warp - 4;
+        const int quad = warp & 3, acc = ew >> 2;
+        const int row = acc * 128 + quad * 32 + lane;
+        const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kMaxHidden);
+        const float bias2 = *p.b2;
+        float sum_rh[kMaxHidden / 32], sum_p[kMaxHidden / 32];   // lane l: columns c0 + l of this warp's rows
+#pragma unroll
+        for (int c = 0; c < kMaxHidden / 32; ++c) sum_rh[c] = sum_p[c] = 0.0f;
+        float sum_r = 0.0f;
+        int it = 0;
+        for (unsigned int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
+            if (!mbar_wait(&tp->acc_full, (uint32_t)(it & 1), abort_flag)) {
+                if (lane == 0) step_give_up(p, tp);
+                break;
+            }
+            tc_fence_after_sync();
+            const int64_t i = (int64_t)tile * kSuperRows + row;
+            // this row's loss and validity are requested before the pass over TMEM
+            bool valid = i < m;
+            float f_i = 0.0f;
+            if (valid) {
+                f_i = __ldg(p.loss + i);
+                if (GATHER && (unsigned long long)(long long)p.row_idx[i] >= (unsigned long long)p.n_stored) {
+                    latch(p.ctl, AA_ERR_BAD_INDEX);
+                    valid = false;
+                }
+            }
+            float s = 0.0f;
+            for (int c0 = 0; c0 < hidden; c0 += 32) {
+                uint32_t a[32];
+                tmem_ld_32cols(t_row + (uint32_t)c0, a);
+                tmem_ld_wait();
+#pragma unroll
+                for (int q = 0; q < 32; ++q) s = fmaf(fmaxf(__uint_as_float(a[q]) + b1_s[c0 + q], 0.0f), w2_s[c0 + q], s);
+            }
+            float r = 0.0f;
+            if (valid) {
+                const float z = (double)f_i > T_shrink ? 1.0f : 0.0f;
+                r = sigmoid_f32(s + bias2) - z;
+            }
+            sum_r += r;
+            const __nv_bfloat16 r_bf = __float2bfloat16_rn(r);
+            const __nv_bfloat16 zero_bf = __float2bfloat16_rn(0.0f);
+#pragma unroll
+            for (int c = 0; c < kMaxHidden / 32; ++c) {
+                const int c0 = c * 32;
+                if (c0 < hidden) {
+                    uint32_t a[32];
+                    tmem_ld_32cols(t_row + (uint32_t)c0, a);
+                    tmem_ld_wait();
+                    float rh[32], pm[32];
+#pragma unroll
+                    for (int q = 0; q < 32; ++q) {
+                        const float pre = __uint_as_float(a[q]) + b1_s[c0 + q];
+                        const bool on = pre > 0.0f;
+                        rh[q] = on ? r * pre : 0.0f;
+                        pm[q] = on ? r : 0.0f;
+                        // P^T[u][i]: the warp's 32 rows are adjacent in i
+                        p.Pt[(int64_t)(c0 + q) * p.pitch + i] = on ? r_bf : zero_bf;
+                    }
+                    sum_rh[c] += lanes_transpose_sum(rh, lane);
+                    sum_p[c] += lanes_transpose_sum(pm, lane);
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tp->acc_empty);
+        }
+#pragma unroll
+        for (int c = 0; c < kMaxHidden / 32; ++c) {
+            col_s[(ew * 2 + 0) * kMaxHidden + c * 32 + lane] = sum_rh[c];
+            col_s[(ew * 2 + 1) * kMaxHidden + c * 32 + lane] = sum_p[c];
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum_r += __shfl_xor_sync(0xFFFFFFFFu, sum_r, o);
+        if (lane == 0) rsum_s[ew] = sum_r;
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    if (warp == 2) tmem_dealloc(tmem_base, kTmemCols);
+    // this CTA's column sums, warps added in a fixed order
+    float* out = p.small + (int64_t)blockIdx.x * (2 * kMaxHidden + 1);
+    for (int j = tid; j < 2 * kMaxHidden; j += kStepMlpThreads) {
+        const int which = j / kMaxHidden, u = j % kMaxHidden;
+        float t = 0.0f;
+        for (int w = 0; w < kStepEpiWarps; ++w) t += col_s[(w * 2 + which) * kMaxHidden + u];
+        out[j] = t;
+    }
+    if (tid == 0) {
+        float t = 0.0f;
+        for (int w = 0; w < kStepEpiWarps; ++w) t += rsum_s[w];
+        out[2 * kMaxHidden] = t;
+    }
+}
+
+// ---------------------------------------------------------------- G = P^T X over the batch rows
+struct GradPipe {
+    uint64_t full[kMlpStages], empty[kMlpStages];
+    uint64_t acc_full, drain;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+template <bool GATHER>
+__global__ void __launch_bounds__(kStepMlpThreads, 1)
+mlp_w1_grad_kernel(const __grid_constant__ CUtensorMap map_pt, const __grid_constant__ CUtensorMap map_x, MlpStepParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* ring = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    constexpr uint32_t kPtBytes = kMaxHidden * 128;                 // P^T slice: up to 256 hidden rows x 64 batch positions
+    constexpr uint32_t kXChunkBytes = kRowSlice * 128;              // 64 batch rows x 64 feature columns
+    constexpr uint32_t kStage = kPtBytes + 4 * kXChunkBytes;        // 64 KB
+    GradPipe* gp = reinterpret_cast<GradPipe*>(ring + (size_t)kMlpStages * kStage);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int s = 0; s < kMlpStages; ++s) {
+            mbar_init(&gp->full[s], 1);
+            mbar_init(&gp->empty[s], 1);
+        }
+        mbar_init(&gp->acc_full, 1);
+        mbar_init(&gp->drain, 1);
+        gp->abort_flag = 0;
+        mbar_fence_init();
+        prefetch_tensormap(&map_pt);
+        prefetch_tensormap(&map_x);
+    }
+    if (warp == 2) tmem_alloc(&gp->tmem_base, kTmemCols);
+    volatile int* abort_flag = &gp->abort_flag;
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *(volatile uint32_t*)&gp->tmem_base;
+
+    const int64_t m = mlp_batch_size(p);
+    const int chunk = blockIdx.x % p.n_chunks, split = blockIdx.x / p.n_chunks;
+    const int64_t total_slices = (m + kRowSlice - 1) / kRowSlice;
+    const int64_t per = (total_slices + p.splits - 1) / p.splits;
+    const int64_t s_begin = (int64_t)split * per;
+    const int64_t s_end = s_begin + per < total_slices ? s_begin + per : total_slices;
+    const int n_slices = s_end > s_begin ? (int)(s_end - s_begin) : 0;
+    const int col0 = chunk * kFeatChunk;
+    int n_q = (int)((p.d - col0 + 63) / 64);           // 64-column feature chunks that exist
+    if (n_q > 4) n_q = 4;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer
+        int stage = 0, j = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        const int grp = lane & 15, half = lane >> 4;
+        for (int sl = 0; sl < n_slices; ++sl) {
+            const int64_t i0 = (s_begin + sl) * kRowSlice;
+            int r0 = 0, r1 = 0, r2 = 0, r3 = 0;
+            if (GATHER) {
+                int rr[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int64_t i = i0 + grp * 4 + q;
+                    long long row = i < m ? (long long)p.row_idx[i] : 0;
+                    if ((unsigned long long)row >= (unsigned long long)p.n_stored) row = 0;   // its P column is zero
+                    rr[q] = (int)row;
+                }
+                r0 = rr[0]; r1 = rr[1]; r2 = rr[2]; r3 = rr[3];
+            }
+            if (!mbar_wait(&gp->empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
+            unsigned char* pt_dst = ring + (size_t)stage * kStage;
+            unsigned char* x_dst = pt_dst + kPtBytes;
+            if (lane == 0) {
+                mbar_arrive_expect_tx(&gp->full[stage], p.g.b_bytes + (uint32_t)n_q * kXChunkBytes);   // P^T box: hidden rows
+                tma_load_2d(pt_dst, &map_pt, (int)i0, 0, &gp->full[stage]);
+                if (!GATHER)
+                    for (int q = 0; q < n_q; ++q) tma_load_2d(x_dst + q * kXChunkBytes, &map_x, col0 + q * 64, (int)i0, &gp->full[stage]);
+            }
+            if (GATHER) {
+                __syncwarp();
+#pragma unroll
+                for (int cq = 0; cq < 2; ++cq) {
+                    const int q = half * 2 + cq;
+                    if (q < n_q) tma_gather4(x_dst + q * kXChunkBytes + (grp * 4) * 128, &map_x, col0 + q * 64, r0, r1, r2, r3, &gp->full[stage]);
+                }
+            }
+            __syncwarp();
+            ++j;
+            if (++stage == kMlpStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) {
+            if (lane == 0) { latch(p.ctl, AA_ERR_SCAN_TIMEOUT); *abort_flag = 1; }
+            const int pending = j < kMlpStages ? j : kMlpStages;
+            for (int back = 1; back <= pending; ++back) {
+                const int jj = j - back, st = jj % kMlpStages, use = jj / kMlpStages;
+                const long long t0 = clock64();
+                while (!mbar_try_wait(&gp->full[st], (uint32_t)(use & 1)) && clock64() - t0 < kWaitCycles) {}
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        const uint32_t idesc = umma_idesc_bf16(128, kFeatChunk, false, true);   // A = P^T K-major, B = feature rows MN-major
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int sl = 0; sl < n_slices; ++sl) {
+            if (!mbar_wait(&gp->full[stage], phase, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            if (lane == 0) {
+                const uint32_t a_addr = smem_u32(ring + (size_t)stage * kStage);
+                const uint32_t b_addr = a_addr + kPtBytes;
+#pragma unroll
+                for (int k = 0; k < kRowSlice / 16; ++k) {
+                    // 16 batch rows = two 8-row groups (1024 bytes apart); 64-column chunks are 8192 bytes apart
+                    const uint64_t b_desc = umma_smem_desc(b_addr + k * 2048, kXChunkBytes, 1024);
+                    const bool acc = (sl | k) != 0;
+                    umma_bf16(tmem_base, umma_smem_desc(a_addr + k * 32, 16, 1024), b_desc, idesc, acc);
+                    umma_bf16(tmem_base + kFeatChunk, umma_smem_desc(a_addr + 128 * 128 + k * 32, 16, 1024), b_desc, idesc, acc);
+                }
+                umma_commit(&gp->empty[stage]);
+                if (sl == n_slices - 1) umma_commit(&gp->acc_full);
+            }
+            __syncwarp();
+            if (++stage == kMlpStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok && lane == 0) { latch(p.ctl, AA_ERR_SCAN_TIMEOUT); *abort_flag = 1; }
+        if (lane == 0) umma_commit(&gp->drain);
+        __syncwarp();
+        const long long t0 = clock64();
+        while (!mbar_try_wait(&gp->drain, 0) && clock64() - t0 < kWaitCycles) {}
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------ epilogue: this CTA's partial of G
+        const int quad = warp & 3, acc = (warp - 4) >> 2;
+        const int u = acc * 128 + quad * 32 + lane;                 // hidden unit
+        const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kFeatChunk);
+        bool have = n_slices > 0;
+        if (have && !mbar_wait(&gp->acc_full, 0, abort_flag)) {
+            if (lane == 0) { latch(p.ctl, AA_ERR_SCAN_TIMEOUT); *abort_flag = 1; }
+            have = false;
+        }
+        tc_fence_after_sync();
+        float* dst = p.part + ((int64_t)split * p.g.hidden + u) * p.d_pad + col0;
+        for (int c0 = 0; c0 < kFeatChunk; c0 += 32) {
+            uint32_t v[32];
+            if (have) {
+                tmem_ld_32cols(t_row + (uint32_t)c0, v);
+                tmem_ld_wait();
+            } else {
+#pragma unroll
+                for (int q = 0; q < 32; ++q) v[q] = 0u;
+            }
+            if (u < p.g.hidden && col0 + c0 < p.d_pad) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    reinterpret_cast<float4*>(dst + c0)[q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
+                                                                        __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+            }
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    if (warp == 2) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+// ---------------------------------------------------------------- updates
+__global__ void __launch_bounds__(256) mlp_apply_w1_kernel(MlpStepParams p) {
+    const int64_t m = mlp_batch_size(p);
+    if (m <= 0) return;
+    const int64_t total = (int64_t)p.g.hidden * p.d;
+    const float scale = p.lr / (float)m;
+    for (int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; q < total; q += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t u = q / p.d, k = q - u * p.d;
+        float g = 0.0f;
+        for (int s = 0; s < p.splits; ++s) g += p.part[((int64_t)s * p.g.hidden + u) * p.d_pad + k];
+        const float w = p.W1[q] - scale * __ldg(p.w2 + u) * g;
+        p.W1[q] = w;
+        p.W1_bf16[q] = __float2bfloat16_rn(w);
+    }
+}
+
+__global__ void __launch_bounds__(kMaxHidden) mlp_apply_small_kernel(MlpStepParams p, int ctas) {
+    const int64_t m = mlp_batch_size(p);
+    if (m <= 0) return;
+    const float scale = p.lr / (float)m;
+    const int u = threadIdx.x;
+    if (u < p.g.hidden) {
+        float g_w2 = 0.0f, g_b1 = 0.0f;
+        for (int c = 0; c < ctas; ++c) {
+            const float* in = p.small + (int64_t)c * (2 * kMaxHidden + 1);
+            g_w2 += in[u];
+            g_b1 += in[kMaxHidden + u];
+        }
+        const float w2_old = p.w2[u];
+        p.b1[u] = p.b1[u] - scale * w2_old * g_b1;
+        p.w2[u] = w2_old - scale * g_w2;
+    }
+    if (u == 0) {
+        float g_b2 = 0.0f;
+        for (int c = 0; c < ctas; ++c) g_b2 += p.small[(int64_t)c * (2 * kMaxHidden + 1) + 2 * kMaxHidden];
+        p.b2[0] = p.b2[0] - scale * g_b2;
+    }
+}
+
+}  // namespace
+
+size_t mlp_step_workspace_bytes(int64_t max_rows, int64_t max_d, int64_t max_hidden, size_t* pt_bytes, size_t* small_bytes) {
+    const size_t pitch = (size_t)((max_rows + kSuperRows - 1) / kSuperRows * kSuperRows);
+    *pt_bytes = ((size_t)max_hidden * pitch * 2 + 255) / 256 * 256;
+    *small_bytes = ((size_t)kMaxMlpCtas * (2 * kMaxHidden + 1) * 4 + 255) / 256 * 256;
+    // split-K partials: chunks * splits <= kMaxMlpCtas CTAs, each [hidden x 256] fp32 (+ one chunk of slack per split row)
+    const size_t d_pad = (size_t)((max_d + kFeatChunk - 1) / kFeatChunk * kFeatChunk);
+    const size_t n_chunks = d_pad / kFeatChunk;
+    size_t splits = kMaxMlpCtas / n_chunks;
+    if (splits < 1) splits = 1;
+    return splits * (size_t)max_hidden * d_pad * 4;
+}
+
+aa_status launch_assistant_step_mlp(aa_ctx_impl* c, const MlpFeat& f, float* W1_master, const int32_t* row_idx, int64_t n_stored,
+                                    int64_t m_host, const int32_t* count_dev, const float* loss, float lr, int thresh_mode,
+                                    float threshold) {
+    if (m_host <= 0) return AA_OK;
+    if (f.hidden < 16 || f.hidden > kMaxHidden || f.hidden % 16) return AA_ERR_UNSUPPORTED;
+    if ((uintptr_t)f.x % 16 || (f.row_stride * 2) % 16 || (uintptr_t)f.W1_bf16 % 16 || (f.d * 2) % 16) return AA_ERR_UNSUPPORTED;
+    if (!c->mlp_pt || m_host > c->max_rows || f.d > c->max_d || f.hidden > c->max_hidden) return AA_ERR_WORKSPACE;
+    const bool gather = row_idx != nullptr;
+    MlpStepParams p = {};
+    p.row_idx = row_idx;
+    p.n_stored = n_stored;
+    p.m_host = m_host;
+    p.count_dev = count_dev;
+    p.loss = loss;
+    p.thresh_mode = thresh_mode;
+    p.threshold = threshold;
+    p.lr = lr;
+    p.W1 = W1_master;
+    p.W1_bf16 = static_cast<__nv_bfloat16*>(const_cast<void*>(f.W1_bf16));
+    p.b1 = const_cast<float*>(f.b1);
+    p.w2 = const_cast<float*>(f.w2);
+    p.b2 = const_cast<float*>(f.b2);
+    p.d = f.d;
+    p.g = make_mlp_geom(f.d, f.hidden);
+    p.Pt = static_cast<__nv_bfloat16*>(c->mlp_pt);
+    p.pitch = (m_host + kSuperRows - 1) / kSuperRows * kSuperRows;
+    p.small = c->mlp_small;
+    p.part = c->mlp_part;
+    p.d_pad = (f.d + kFeatChunk - 1) / kFeatChunk * kFeatChunk;
+    p.n_chunks = (int)(p.d_pad / kFeatChunk);
+    p.ctl = c->ctl;
+    int max_ctas = c->sm_count < kMaxMlpCtas ? c->sm_count : kMaxMlpCtas;
+    if (p.n_chunks > max_ctas) return AA_ERR_UNSUPPORTED;
+    const int64_t slices = (m_host + kRowSlice - 1) / kRowSlice;
+    int64_t splits = max_ctas / p.n_chunks;
+    if (splits > slices) splits = slices;
+    if (splits < 1) splits = 1;
+    while (splits > 1 && (size_t)splits * (size_t)f.hidden * (size_t)p.d_pad * 4 > c->mlp_part_bytes) --splits;
+    if ((size_t)splits * (size_t)f.hidden * (size_t)p.d_pad * 4 > c->mlp_part_bytes) return AA_ERR_WORKSPACE;
+    p.splits = (int)splits;
+
+    alignas(64) CUtensorMap map_x, map_w, map_pt, map_xg;
+    if (!encode_bf16_tile_map(&map_x, f.x, (uint64_t)f.n, (uint64_t)f.d, (uint64_t)f.row_stride, gather ? 1 : kSuperRows) ||
+        !encode_bf16_tile_map(&map_w, f.W1_bf16, (uint64_t)f.hidden, (uint64_t)f.d, (uint64_t)f.d, (uint32_t)f.hidden) ||
+        !encode_bf16_tile_map(&map_pt, p.Pt, (uint64_t)f.hidden, (uint64_t)p.pitch, (uint64_t)p.pitch, (uint32_t)f.hidden) ||
+        !encode_bf16_tile_map(&map_xg, f.x, (uint64_t)f.n, (uint64_t)f.d, (uint64_t)f.row_stride, gather ? 1 : kRowSlice))
+        return AA_ERR_CUDA;
+
+    // 1. forward + residuals + P^T
+    {
+        const size_t smem = 1024 + (size_t)kMlpStages * p.g.stage_bytes + sizeof(float) * (2 * kMaxHidden + kStepEpiWarps * 2 * kMaxHidden) +
+                            sizeof(double) * (kStepMlpThreads / 32) + sizeof(float) * kStepEpiWarps + sizeof(TilePipe) + 64;
+        const void* kernel = gather ? (const void*)mlp_residual_kernel<true> : (const void*)mlp_residual_kernel<false>;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return AA_ERR_CUDA;
+        const int64_t tiles = (m_host + kSuperRows - 1) / kSuperRows;
+        int grid = max_ctas;
+        if (grid > tiles) grid = (int)tiles;
+        void* args[] = {&map_x, &map_w, &p};
+        if (cudaLaunchKernel(kernel, dim3(grid), dim3(kStepMlpThreads), args, smem, c->stream) != cudaSuccess) return AA_ERR_CUDA;
+        ++c->launches;
+        // 2. G = P^T X
+        const size_t smem2 = 1024 + (size_t)kMlpStages * (kMaxHidden * 128 + 4 * kRowSlice * 128) + sizeof(GradPipe) + 64;
+        const void* k2 = gather ? (const void*)mlp_w1_grad_kernel<true> : (const void*)mlp_w1_grad_kernel<false>;
+        if (cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2) != cudaSuccess) return AA_ERR_CUDA;
+        void* args2[] = {&map_pt, &map_xg, &p};
+        if (cudaLaunchKernel(k2, dim3(p.n_chunks * p.splits), dim3(kStepMlpThreads), args2, smem2, c->stream) != cudaSuccess)
+            return AA_ERR_CUDA;
+        ++c->launches;
+        // 3. updates (W1 first: it reads the old w2)
+        void* args3[] = {&p};
+        const int64_t total = f.hidden * f.d;
+        int agrid = (int)((total + 255) / 256);
+        if (agrid > c->sm_count * 8) agrid = c->sm_count * 8;
+        if (cudaLaunchKernel((const void*)mlp_apply_w1_kernel, dim3(agrid), dim3(256), args3, 0, c->stream) != cudaSuccess) return AA_ERR_CUDA;
+        ++c->launches;
+        void* args4[] = {&p, &grid};
+        if (cudaLaunchKernel((const void*)mlp_apply_small_kernel, dim3(1), dim3(kMaxHidden), args4, 0, c->stream) != cudaSuccess)
+            return AA_ERR_CUDA;
+        ++c->launches;
+    }
+    return AA_OK;
+}
+
+}  // namespace aa

@@ -158,6 +158,78 @@ def test_mlp_candidate_list_gathers_rows(aa):
     assert aa.aa_device_status() == B.AA_ERR_BAD_INDEX
 
 
+def params_close(got, ref, what, slack=None):
+    ref = np.asarray(ref, np.float64).reshape(-1)
+    got = np.asarray(got, np.float64).reshape(-1)
+    tol = 1e-4 * np.abs(ref) + 1e-4 * math.sqrt(float(np.mean(ref ** 2)) + 1e-300)
+    if slack is not None:
+        tol = tol + slack
+    err = np.abs(got - ref)
+    assert np.all(err <= tol), (what, float(np.max(err - tol)))
+
+
+@pytest.mark.parametrize("n,m,d,hidden,use_rows,thr,lr", [
+    (300, 300, 64, 16, False, None, 0.1), (2000, 1500, 192, 64, True, None, 0.1), (1000, 1000, 200, 256, False, 1.5, 0.1),
+    (5000, 2777, 3072, 256, True, None, 0.05), (700, 1, 128, 32, True, None, 0.1), (1300, 1300, 600, 128, False, None, 1.0),
+])
+def test_mlp_assistant_step(aa, n, m, d, hidden, use_rows, thr, lr):
+    rng = np.random.default_rng(n + d)
+    x = W.normal((n, d), 1.0, 60 + d, torch.bfloat16, DEV)
+    W1, W1b, b1, w2, b2 = make_mlp(d, hidden, 61 + d)
+    loss = (W.normal((m,), 1.0, 62, torch.float32, DEV).abs() * 2).contiguous()
+    rows = np.sort(rng.permutation(n)[:m]).astype(np.int32) if use_rows else None
+    rows_t = None if rows is None else torch.from_numpy(rows).to(DEV)
+    host = {k: v.cpu().numpy().copy() for k, v in (("W1", W1), ("b1", b1), ("w2", w2))}
+    b2_0 = float(b2.item())
+    W1b_bits = W.to_oracle(W1b).copy()
+    feat = B.dense_features(x, row_idx=rows_t) if use_rows else B.dense_features(x[:m])
+    cnt = torch.tensor([m], dtype=torch.int32, device=DEV)
+    aa.aa_assistant_step(feat, loss, B.mlp_assistant(W1, W1b, b1, w2, b2), lr, threshold=thr, count_dev=cnt)
+    torch.cuda.synchronize()
+    assert aa.aa_device_status() == B.AA_OK
+    ref = O.assistant_step_mlp(W.to_oracle(x), loss.cpu().numpy(), host["W1"], W1b_bits, host["b1"], host["w2"], b2_0, lr,
+                               T=thr, row_idx=rows)
+    # P = r [a > 0] goes through the tensor cores in bf16 (relative rounding 2^-9 per term), and a pre-activation
+    # within 1e-4 of zero may switch its unit on or off: bound of what that does to the W1 gradient
+    gW1 = ref["grads"][0]
+    xs = (bf16_values(x) if rows is None else bf16_values(x)[rows])[:m]
+    r = O.sigmoid(ref["s"]) - ref["z"]
+    on = ref["a"] > 0
+    near = np.abs(ref["a"]) < 1e-4
+    w2h = host["w2"].astype(np.float64)
+    bound = (np.abs(r)[:, None] * on).T @ np.abs(xs) * np.abs(w2h)[:, None] / m * 2.0 ** -8
+    bound += (np.abs(r)[:, None] * near).T @ np.abs(xs) * np.abs(w2h)[:, None] / m
+    # parameters after the update: rel 1e-4 (+ 1e-4 rms floor).  At the step sizes the workloads use (lr <= 0.1) and
+    # batches of a thousand rows or more the bf16 rounding of P is far below that bar; for a tiny batch or a step
+    # size near 1 the update itself is a large fraction of the weight and the bf16 term is allowed for explicitly.
+    plain = m >= 1000 and lr <= 0.1
+    params_close(W1.cpu().numpy(), ref["W1"], "W1", slack=None if plain else lr * bound.reshape(-1))
+    params_close(b1.cpu().numpy(), ref["b1"], "b1")
+    params_close(w2.cpu().numpy(), ref["w2"], "w2")
+    params_close([b2.item()], [ref["b2"]], "b2")
+    # the bf16 copy is the nearest-even rounding of the GPU's own new master
+    assert np.array_equal(W.to_oracle(W1b), O.round_bf16(W1.cpu().numpy()))
+    assert np.abs(W1.cpu().numpy() - host["W1"]).max() > 0
+    # the gradient itself, recovered from the update (which is rounded once to fp32)
+    g_gpu = (host["W1"].astype(np.float64) - W1.double().cpu().numpy()) / lr
+    ulp = np.abs(host["W1"]) * 2.0 ** -23 / lr
+    assert np.all(np.abs(g_gpu - gW1) <= bound + 2 * ulp + 1e-12), float(np.max(np.abs(g_gpu - gW1) - bound - 2 * ulp))
+
+
+def test_mlp_step_empty_batch_and_zero_lr(aa):
+    x = W.normal((400, 64), 1.0, 1, torch.bfloat16, DEV)
+    W1, W1b, b1, w2, b2 = make_mlp(64, 32, 2)
+    before = [t.clone() for t in (W1, W1b, b1, w2, b2)]
+    loss = torch.ones(400, device=DEV)
+    zero = torch.zeros(1, dtype=torch.int32, device=DEV)
+    asst = B.mlp_assistant(W1, W1b, b1, w2, b2)
+    aa.aa_assistant_step(B.dense_features(x), loss, asst, 0.5, count_dev=zero)
+    aa.aa_assistant_step(B.dense_features(x), loss, asst, 0.0)
+    torch.cuda.synchronize()
+    for t, t0 in zip((W1, W1b, b1, w2, b2), before):
+        assert torch.equal(t, t0)
+
+
 def test_mlp_full_size_pool_sampled(aa):
     """The MLP shape at full size (262,144 x 3072, hidden 256) in the launch configuration that is timed."""
     cfg = W.MlpShape()
