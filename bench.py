@@ -39,8 +39,10 @@ def parse_args():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--pools", type=int, default=8, help="distinct resident pools rotated through the steps")
     ap.add_argument("--e2e-steps", type=int, default=20)
-    ap.add_argument("--cpu-steps", type=int, default=4, help="oracle steps timed for cpu_baseline (0 = skip)")
+    ap.add_argument("--cpu-steps", type=int, default=40, help="oracle steps timed for cpu_baseline (0 = skip)")
     ap.add_argument("--pool-rows", type=int, default=None, help="override the pool size (testing only)")
+    ap.add_argument("--workload", default="image", choices=["image", "mlp"],
+                    help="image = the benchmark workload; mlp = the two-layer (tensor-core) Assistant shape")
     ap.add_argument("--loss-reps", type=int, default=20,
                     help="timed calls of the per-sentence loss on the translation shape (0 = skip)")
     return ap.parse_args()
@@ -413,10 +415,111 @@ def run_b200(args, cfg):
         dist.destroy_process_group()
 
 
+def measured_peak_tflops(sustained: bool):
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            rec = json.load(f)
+        return float(rec["bf16_tflops_sustained" if sustained else "bf16_tflops"]), "measured"
+    except Exception:
+        return (1400.0 if sustained else 1590.0), "fallback"
+
+
+def run_mlp(args):
+    """Secondary workload (--workload mlp): the two-layer Assistant shape, whose scoring is a dense bf16 contraction.
+    One step = MLP score+shrink+compact, 1000-class instance loss, MLP Assistant step on the accepted rows."""
+    import torch
+
+    from paper_1905_03381_b200 import binding as B, build as lib_build, workloads as W
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    lib_build.build()
+    cfg = W.MlpShape()
+    if args.pool_rows:
+        cfg.n = args.pool_rows
+    x = cfg.pool(dev)
+    W1, b1, w2, b2 = cfg.assistant(dev)
+    W1b = W1.to(torch.bfloat16).contiguous()
+    logits = cfg.logits(cfg.n, dev)
+    labels = cfg.labels(cfg.n, dev)
+    aa = B.AutoAssist(max_rows=cfg.n, max_d=cfg.d, max_hidden=cfg.hidden, device=dev)
+    asst = B.mlp_assistant(W1, W1b, b1, w2, b2)
+    out_idx = torch.zeros(cfg.n, dtype=torch.int32, device=dev)
+    K = args.steps
+    warm = max(args.warmup, 3)
+    counts = torch.zeros(warm + K, dtype=torch.int32, device=dev)
+    loss = torch.zeros(cfg.n, dtype=torch.float32, device=dev)
+    feat, batch = B.dense_features(x), B.dense_features(x, row_idx=out_idx)
+    lg = B.logits_desc(logits)
+
+    def step(i, ev=None):
+        cnt = counts[i:i + 1]
+        if ev: ev[0].record()
+        aa.aa_score_shrink(feat, asst, cfg.gamma, cfg.philox_seed, i, out_idx, cnt)
+        if ev: ev[1].record()
+        aa.aa_instance_loss(lg, labels, loss, count_dev=cnt)
+        if ev: ev[2].record()
+        aa.aa_assistant_step(batch, loss, asst, cfg.lr, count_dev=cnt)
+        if ev: ev[3].record()
+
+    for i in range(warm):
+        step(i)
+    torch.cuda.synchronize()
+    assert aa.aa_device_status() == B.AA_OK
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.3)
+    n0 = aa.aa_launch_count()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for i in range(K):
+        step(warm + i, evs[i])
+    t1.record()
+    torch.cuda.synchronize()
+    time.sleep(0.2)
+    sampler.stop()
+    assert aa.aa_device_status() == B.AA_OK
+    ms = t0.elapsed_time(t1) / K
+    score_ms = sum(e[0].elapsed_time(e[1]) for e in evs) / K
+    loss_ms = sum(e[1].elapsed_time(e[2]) for e in evs) / K
+    asst_ms = sum(e[2].elapsed_time(e[3]) for e in evs) / K
+    m_mean = float(counts[warm:].float().mean().item())
+    flops = 2.0 * cfg.n * cfg.d * cfg.hidden
+    peak, kind = measured_peak_tflops(sustained=True)
+    hbm, hkind = measured_peak_gbs()
+    line = {
+        "metric": METRIC, "value": cfg.n / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": K, "warmup": warm,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": f"MLP Assistant shape: pool {cfg.n} x {cfg.d} bf16 N(0,1), {cfg.d}->{cfg.hidden} (ReLU)->1, "
+                               f"{cfg.classes}-class fp32 logits N(0,3), mix {cfg.gamma}, SGD lr {cfg.lr} on both layers",
+                   "l2_policy": "inputs larger than L2 (pool 1.6 GB)"},
+        "roofline": {"bound": "tensor", "kernel": "mlp_score_shrink_kernel", "achieved": flops / (score_ms * 1e-3) / 1e12,
+                     "peak": peak, "unit": "TFLOP/s", "frac": flops / (score_ms * 1e-3) / 1e12 / peak,
+                     "peak_kind": f"of {kind} (sustained cuBLAS bf16)", "traffic": None, "avg_launch_ms": score_ms,
+                     "hbm_GBs": cfg.n * cfg.d * 2 / (score_ms * 1e-3) / 1e9, "hbm_frac": cfg.n * cfg.d * 2 / (score_ms * 1e-3) / 1e9 / hbm},
+        "stages": {"score_shrink": {"ms": score_ms}, "instance_loss": {"ms": loss_ms, "rows_per_s": m_mean / (loss_ms * 1e-3),
+                   "GB/s": m_mean * (cfg.classes * 4 + 8) / (loss_ms * 1e-3) / 1e9},
+                   "assistant_step": {"ms": asst_ms, "TFLOP/s": 2 * 2.0 * m_mean * cfg.d * cfg.hidden / (asst_ms * 1e-3) / 1e12}},
+        "accepted_mean": m_mean, "gpu_launches": int(aa.aa_launch_count() - n0), "clocks": sampler.summary(),
+    }
+    print(json.dumps(line), flush=True)
+    aa.close()
+
+
 def main():
     args = parse_args()
     from paper_1905_03381_b200 import workloads as W
 
+    if args.workload == "mlp":
+        if args.impl == "reference" or args.gpus != 1:
+            raise SystemExit("--workload mlp is a single-GPU measurement of the library only")
+        run_mlp(args)
+        return
     cfg = W.ImageShape()
     if args.pool_rows:
         cfg.n = args.pool_rows
