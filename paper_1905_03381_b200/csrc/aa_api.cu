@@ -20,7 +20,7 @@ struct Layout {
 
 Layout make_layout(int64_t max_rows, int64_t max_d, int64_t max_hidden) {
     Layout L;
-    L.max_tiles = (max_rows + 31) / 32 + 1;
+    L.max_tiles = (max_rows + 15) / 16 + 1;   // the smallest compaction tile is 16 candidates
     size_t off = sizeof(Control);
     L.tile_state_off = off;
     off = align_up(off + sizeof(unsigned long long) * (size_t)L.max_tiles, 256);

@@ -136,7 +136,7 @@ __device__ __forceinline__ void warp_shrink_compact(const ShrinkParams& p, unsig
         if (u < units) {
             const long long k = k0 + u * 32 + lane;
             bool keep = false;
-            if (k < p.n_cand) {
+            if (u * 32 + lane < p.tile_rows && k < p.n_cand) {   // a tile may be shorter than a warp
                 keep = keep_decision(p, k, sv[u]);
                 if (p.out_score) p.out_score[k] = sv[u];
                 if (p.out_mask) p.out_mask[k] = keep ? 1 : 0;

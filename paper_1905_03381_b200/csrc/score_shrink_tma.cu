@@ -1,8 +1,8 @@
 // Assistant score -> Bernoulli shrink -> ordered batch list for 16-byte aligned dense rows,
 // as one persistent, warp-specialised CTA per SM fed by bulk asynchronous copies.
 //
-//   producer warp : takes tile tickets (the next one is requested while the current tile is
-//                   being issued) and streams the tile's rows into a shared-memory ring with
+//   producer warp : starts on tile blockIdx.x, then takes tile tickets (the next one is requested
+//                   a few stages before the current tile ends) and streams the tile's rows into a shared-memory ring with
 //                   cp.async.bulk (one copy per stage of contiguous rows, or one per row when a
 //                   candidate list gathers rows); it runs ahead of the consumers by the depth of
 //                   the ring, across tile boundaries.  Its per-stage work is a handful of
@@ -46,6 +46,7 @@ struct TmaGeometry {
     int split;             // consumer warps sharing one stage (1 or 2)
     int contiguous;        // rows of a chunk are adjacent in memory: one copy per chunk
     int nvec;              // 16-byte vectors per row
+    int slot_rows;         // floats reserved per score slot (tile rows rounded up to a warp)
     uint32_t row_bytes;
 };
 
@@ -157,7 +158,7 @@ __global__ void __launch_bounds__(kTmaThreads, 1) score_shrink_tma_kernel(DenseF
     unsigned char* x_ring = smem;
     float* w_s = reinterpret_cast<float*>(smem + (size_t)g.stages * g.stage_bytes);
     float* s_ring = w_s + (size_t)g.nvec * VE;
-    RingControl* cb = reinterpret_cast<RingControl*>(s_ring + kScoreSlots * kMaxTmaTileRows);
+    RingControl* cb = reinterpret_cast<RingControl*>(s_ring + kScoreSlots * g.slot_rows);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cpt = 1 << g.cpt_shift;   // chunks (ring stages' worth of rows) per tile
@@ -194,13 +195,16 @@ __global__ void __launch_bounds__(kTmaThreads, 1) score_shrink_tma_kernel(DenseF
         int j = 0, q = 0, stage = 0;
         uint32_t phase = 0;   // parity of the current pass over the ring
         bool ok = true;
-        unsigned int next_tile = 0;
-        if (lane == 0) next_tile = atomicAdd(&p.ctl->ticket, 1u);
-        next_tile = __shfl_sync(0xFFFFFFFFu, next_tile, 0);
+        // The first tile of a CTA is its block index (no round trip before the first copy); later
+        // tiles come from the ticket counter, which therefore counts from gridDim.x.  The next ticket
+        // is requested only a few stages before this tile's last copy is issued, just early enough to
+        // hide the atomic: a CTA never holds more than the tile it is streaming, which keeps the
+        // CTAs' finishing times close together.
+        const int req_c = cpt > 3 ? cpt - 3 : 0;
+        unsigned int next_tile = blockIdx.x;
         while (ok) {
             const unsigned int tile = next_tile;
             if (tile >= p.n_tiles) break;
-            if (lane == 0) next_tile = atomicAdd(&p.ctl->ticket, 1u);   // lands while this tile is issued
             const int slot = q & (kScoreSlots - 1);
             // the tail has released this score slot (it also guards the slot's tile record)
             if (q >= kScoreSlots && !mbar_wait(&cb->s_empty[slot], (uint32_t)(((q >> kSlotShift) - 1) & 1), abort_flag)) { ok = false; break; }
@@ -209,6 +213,7 @@ __global__ void __launch_bounds__(kTmaThreads, 1) score_shrink_tma_kernel(DenseF
             long long rows_left = p.n_cand - k_tile;   // > 0
             const unsigned char* src = base + (size_t)k_tile * stride_bytes;
             for (int c = 0; c < cpt; ++c) {
+                if (c == req_c && lane == 0) next_tile = gridDim.x + atomicAdd(&p.ctl->ticket, 1u);
                 if (j >= g.stages && !mbar_wait(&cb->x_empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
                 unsigned char* dst = x_ring + (size_t)stage * g.stage_bytes;
                 if (g.contiguous) {
@@ -289,7 +294,7 @@ __global__ void __launch_bounds__(kTmaThreads, 1) score_shrink_tma_kernel(DenseF
                 if (j >= *(volatile int*)&cb->stop_j) break;
                 const int chunk = j & (cpt - 1), slot = (j >> g.cpt_shift) & (kScoreSlots - 1);
                 consume_rows<T, LPR>(xs, w_s, rows_per, g.nvec, g.row_bytes, bias,
-                                     s_ring + slot * kMaxTmaTileRows + chunk * g.chunk_rows + part * rows_per, lane);
+                                     s_ring + slot * g.slot_rows + chunk * g.chunk_rows + part * rows_per, lane);
                 __syncwarp();
                 if (lane == 0) {
                     mbar_arrive(&cb->s_full[slot]);
@@ -299,7 +304,7 @@ __global__ void __launch_bounds__(kTmaThreads, 1) score_shrink_tma_kernel(DenseF
         }
     } else {
         // ------------------------------------------------------------ tail
-        const int units = p.tile_rows >> 5;
+        const int units = (p.tile_rows + 31) >> 5;
         for (int q = warp - (kConsumers + 1);; q += kTails) {
             const int slot = q & (kScoreSlots - 1);
             if (!mbar_wait(&cb->s_full[slot], (uint32_t)((q >> kSlotShift) & 1), abort_flag)) {
@@ -310,7 +315,7 @@ __global__ void __launch_bounds__(kTmaThreads, 1) score_shrink_tma_kernel(DenseF
             const unsigned int tile = cb->tile_of_slot[slot];
             float sv[kMaxUnits];
 #pragma unroll
-            for (int u = 0; u < kMaxUnits; ++u) sv[u] = u < units ? s_ring[slot * kMaxTmaTileRows + u * 32 + lane] : 0.0f;
+            for (int u = 0; u < kMaxUnits; ++u) sv[u] = u < units ? s_ring[slot * g.slot_rows + u * 32 + lane] : 0.0f;
             __syncwarp();
             if (lane == 0) mbar_arrive(&cb->s_empty[slot]);
             warp_shrink_compact<kMaxUnits>(p, tile, epoch, units, sv);
@@ -360,7 +365,9 @@ aa_status launch_score_shrink_dense_tma(aa_ctx_impl* c, const DenseFeat& f_in, S
     if (lpr < 4) lpr = 4;
     if (32 / lpr > rows_per) lpr = 32 / rows_per;
 
-    // tile = one look-back unit: enough rows for ~128 KB, at least 32, a multiple of the chunk
+    // tile = one look-back unit and one ticket: enough rows for ~128 KB, at least 32, a multiple of the
+    // chunk.  (Shorter tiles would even out the CTAs' finishing times, but the look-back then costs more
+    // than it saves: 16-row tiles measured 10 % slower at 65,536 x 3072 bf16.)
     int units = 1;
     while (units < kMaxUnits && (int64_t)units * 32 * row_bytes < 128 * 1024) units <<= 1;
     while (units > 1 && sp.n_cand / (units * 32) < 4 * (int64_t)c->sm_count) units >>= 1;
@@ -369,7 +376,8 @@ aa_status launch_score_shrink_dense_tma(aa_ctx_impl* c, const DenseFeat& f_in, S
     g.cpt_shift = 0;
     while ((1 << g.cpt_shift) < cpt) ++g.cpt_shift;
 
-    const size_t fixed = (size_t)g.nvec * ve * sizeof(float) + sizeof(float) * kScoreSlots * kMaxTmaTileRows + sizeof(RingControl) + 128;
+    g.slot_rows = (tile_rows + 31) / 32 * 32;
+    const size_t fixed = (size_t)g.nvec * ve * sizeof(float) + sizeof(float) * kScoreSlots * g.slot_rows + sizeof(RingControl) + 128;
     const size_t budget = 220 * 1024;
     if (fixed + 2 * (size_t)g.stage_bytes > budget) return AA_ERR_UNSUPPORTED;
     int stages = (int)((budget - fixed) / g.stage_bytes);
