@@ -33,14 +33,29 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
+// Same test, but the hardware may park the thread for up to `hint_ns` while the phase is pending,
+// instead of returning at once: a waiting warp then leaves the issue slots to the warps that work.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint64_t* bar, uint32_t parity, uint32_t hint_ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
+        : "memory");
+    return ok != 0;
+}
+
 constexpr long long kWaitCycles = 2500000000ll;   // ~1.3 s at 1.9 GHz
+constexpr uint32_t kParkNs = 20000;               // longest single park; the abort flag and the clock are checked in between
 
 // Waits for the phase with the given parity.  false = gave up (time limit or abort flag).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait_parked(bar, parity, kParkNs)) return true;
         if (*abort_flag) return false;
         if (clock64() - t0 > kWaitCycles) return false;
     }

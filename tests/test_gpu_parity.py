@@ -318,6 +318,8 @@ def assert_params_close(w_gpu, w_ref):
     (4000, 1777, 3072, torch.bfloat16, True, None), (900, 900, 100, torch.bfloat16, False, 2.0),
     (50, 1, 8, torch.float32, True, None), (600, 600, 7, torch.float32, False, 1.5),
     (400, 333, 4100, torch.float32, True, None), (2000, 2000, 512, torch.float32, False, None),
+    (3000, 3000, 3072, torch.bfloat16, False, None), (1500, 700, 2048, torch.float32, True, 1.0),
+    (900, 900, 2048, torch.bfloat16, False, None), (6000, 5000, 3072, torch.bfloat16, True, None),
 ])
 def test_dense_assistant_step(aa, n, m, d, dtype, use_rows, thr):
     rng = np.random.default_rng(n + d)
