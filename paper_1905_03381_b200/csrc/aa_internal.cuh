@@ -220,6 +220,10 @@ aa_status finish_shrink_params(aa_ctx_impl* c, ShrinkParams& sp, int tile_rows);
 aa_status launch_score_shrink_csr(aa_ctx_impl* c, const CsrFeat& f, ShrinkParams sp);
 aa_status launch_shrink_from_scores(aa_ctx_impl* c, const float* score, ShrinkParams sp);
 
+// Bulk-copy variant for 16-byte aligned rows (writes p.out); AA_ERR_UNSUPPORTED when the shape does not fit.
+struct LossParams;
+aa_status launch_instance_loss_tma(aa_ctx_impl* c, const LossParams& p, int dtype);
+
 aa_status launch_instance_loss(aa_ctx_impl* c, const aa_logits& lg, const int32_t* labels, const int32_t* offsets,
                                int64_t n_seg, const int32_t* count_dev, float* out_loss);
 

@@ -5,103 +5,13 @@
 // t = x * log2(e), so that sum_c 2^(t_c) = S * 2^M; thread states are merged by warp shuffles
 // (and through shared memory when a CTA shares a row).  For sequence tasks the token rows of
 // a sentence are then summed in row order (fp64 accumulator) by a second small kernel.
-#include <math.h>
-
-#include "aa_internal.cuh"
+#include "loss_common.cuh"
 
 namespace aa {
 
 namespace {
 
-constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kRowThreads = 256;   // CTA size when one CTA owns a row
-
-struct LossParams {
-    const void* logits;
-    int64_t rows, cols, row_stride;
-    const int32_t* labels;
-    const int32_t* count_dev;
-    float* out;
-    Control* ctl;
-};
-
-struct RunState {
-    float m;   // running maximum of t = x*log2(e)
-    float s;   // sum of 2^(t - m)
-};
-
-__device__ __forceinline__ void absorb(RunState& st, const float* t, int n) {
-    float vmax = t[0];
-    for (int e = 1; e < n; ++e) vmax = fmaxf(vmax, t[e]);
-    if (vmax > st.m) {
-        st.s *= ex2_approx(st.m - vmax);   // st.m = -inf gives 0 * 0
-        st.m = vmax;
-    }
-    const float ref = st.m == -INFINITY ? 0.0f : st.m;   // all -inf so far: every term is 2^-inf = 0
-    for (int e = 0; e < n; ++e) st.s += ex2_approx(t[e] - ref);
-}
-
-template <int N>
-__device__ __forceinline__ void absorb_vec(RunState& st, const float (&x)[N]) {
-    float t[N];
-#pragma unroll
-    for (int e = 0; e < N; ++e) t[e] = x[e] * kLog2e;
-    float vmax = t[0];
-#pragma unroll
-    for (int e = 1; e < N; ++e) vmax = fmaxf(vmax, t[e]);
-    if (vmax > st.m) {
-        st.s *= ex2_approx(st.m - vmax);
-        st.m = vmax;
-    }
-    const float ref = st.m == -INFINITY ? 0.0f : st.m;
-#pragma unroll
-    for (int e = 0; e < N; ++e) st.s += ex2_approx(t[e] - ref);
-}
-
-__device__ __forceinline__ RunState merge(const RunState& a, const RunState& b) {
-    RunState o;
-    o.m = fmaxf(a.m, b.m);
-    const float ref = o.m == -INFINITY ? 0.0f : o.m;
-    o.s = a.s * ex2_approx(a.m - ref) + b.s * ex2_approx(b.m - ref);
-    return o;
-}
-
-template <int WIDTH>
-__device__ __forceinline__ RunState group_merge(RunState st) {
-#pragma unroll
-    for (int o = WIDTH / 2; o > 0; o >>= 1) {
-        RunState other;
-        other.m = __shfl_xor_sync(0xFFFFFFFFu, st.m, o);
-        other.s = __shfl_xor_sync(0xFFFFFFFFu, st.s, o);
-        st = merge(st, other);
-    }
-    return st;
-}
-
-__device__ __forceinline__ float finish_row(const RunState& st, float label_logit) {
-    return (st.m + lg2_approx(st.s)) * kLn2 - label_logit;
-}
-
-__device__ __forceinline__ int64_t effective_rows(const LossParams& p) {
-    int64_t rows = p.rows;
-    if (p.count_dev) {
-        const int64_t c = *p.count_dev;
-        rows = c < 0 ? 0 : (c < rows ? c : rows);
-    }
-    return rows;
-}
-
-// Label of row r: >= 0 valid; -1 padding or invalid (invalid latches AA_ERR_BAD_INDEX).
-__device__ __forceinline__ int checked_label(const LossParams& p, int64_t r) {
-    const int y = __ldg(p.labels + r);
-    if (y < 0) return -1;
-    if (y >= p.cols) {
-        latch(p.ctl, AA_ERR_BAD_INDEX);
-        return -1;
-    }
-    return y;
-}
 
 // Accumulate the elements [j0, j1) of one row, strided over `nthreads` workers starting at `rank`.
 // Handles any alignment: scalar head up to the first 16-byte boundary, vector body, scalar tail.
@@ -255,7 +165,8 @@ aa_status launch_instance_loss(aa_ctx_impl* c, const aa_logits& lg, const int32_
     p.ctl = c->ctl;
     p.out = offsets ? c->row_scratch : out_loss;
     if (lg.rows > 0) {
-        aa_status st = lg.dtype == AA_BF16 ? launch_rows<uint16_t>(c, p) : launch_rows<float>(c, p);
+        aa_status st = launch_instance_loss_tma(c, p, lg.dtype);
+        if (st == AA_ERR_UNSUPPORTED) st = lg.dtype == AA_BF16 ? launch_rows<uint16_t>(c, p) : launch_rows<float>(c, p);
         if (st != AA_OK) return st;
     }
     if (offsets && n_seg > 0) {

@@ -251,6 +251,24 @@ def test_row_losses(aa, rows, cols, dtype, std):
     assert np.max(np.abs(got - ref)) <= 1e-4, float(np.max(np.abs(got - ref)))
 
 
+@pytest.mark.parametrize("rows,cols,dtype,pad", [
+    (34001, 1000, torch.float32, 0), (17003, 4096, torch.bfloat16, 0), (33000, 1000, torch.float32, 24),
+    (140000, 512, torch.bfloat16, 0), (350001, 100, torch.float32, 0),
+])
+def test_row_losses_large_enough_for_the_bulk_copy_kernel(aa, rows, cols, dtype, pad):
+    """128 MB and more of aligned logit rows of up to 16 KB take the bulk-copy ring kernel."""
+    buf = W.normal((rows, cols + pad), 3.0, rows + cols, dtype, DEV)
+    logits = buf[:, :cols]
+    labels = W.randint(0, cols, (rows,), rows * 3 + cols, DEV)
+    labels[5] = -1                                   # padding row
+    count = rows - 3                                 # device-side row count: the last three rows stay untouched
+    got = run_loss(aa, logits, labels, count=count)
+    ref = O.row_loss(W.to_oracle(logits.contiguous()), labels.cpu().numpy())
+    assert np.max(np.abs(got[:count] - ref[:count])) <= 1e-4, float(np.max(np.abs(got[:count] - ref[:count])))
+    assert got[5] == 0.0 and np.all(got[count:] == -3.0)
+    assert aa.aa_device_status() == B.AA_OK
+
+
 def test_uniform_logits_give_ln_C_on_the_gpu(aa):
     for cols, dtype in ((10, torch.float32), (100, torch.float32), (1000, torch.float32), (32000, torch.bfloat16)):
         logits = torch.full((5, cols), 1.5, dtype=dtype, device=DEV)
