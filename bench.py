@@ -380,7 +380,7 @@ def run_b200(args, cfg):
     peak, peak_kind = measured_peak_gbs()
     alg_bytes = cfg.n * cfg.d * 2 + cfg.d * 4 + accepted * 4 + 4
     achieved = alg_bytes / (score_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "score_shrink_dense_kernel<bf16>", "achieved": achieved, "peak": peak,
+    roofline = {"bound": "hbm", "kernel": "score_shrink_tma_kernel<bf16, 32>", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": ncu_traffic_bytes(cfg.n),
                 "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": score_ms,
                 "frac_of_nominal_8TBs": achieved / 8000.0}
