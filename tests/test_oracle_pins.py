@@ -466,3 +466,38 @@ def test_bf16_rounding_is_nearest_even():
     rnd = np.random.default_rng(16).standard_normal(10000).astype(np.float32)
     ref = torch.from_numpy(rnd).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
     assert np.array_equal(O.round_bf16(rnd), ref)
+
+
+def test_composed_mlp_step_descends_the_objective_to_first_order():
+    """assistant_step_mlp chains score_mlp, labels, mlp_grad, sgd and round_bf16: one small step from parameters whose
+    W1 is exactly representable in bf16 must lower the mean cross-entropy by lr * |grad|^2 to first order, with the
+    gradient taken by central differences of the objective (not by the oracle's own backward pass)."""
+    rng = np.random.default_rng(5)
+    n, d, hidden = 40, 6, 5
+    x = rng.normal(size=(n, d)).astype(np.float32)
+    W1 = (rng.integers(-32, 32, size=(hidden, d)) / 16.0).astype(np.float32)        # bf16-exact values
+    W1_bits = O.round_bf16(W1)
+    b1 = rng.normal(size=hidden).astype(np.float32) * 0.3
+    w2 = rng.normal(size=hidden).astype(np.float32)
+    b2 = np.float32(0.2)
+    f = np.abs(rng.normal(size=n)).astype(np.float32)
+    T = float(np.median(f))
+    z = O.labels(f, T)
+
+    def objective(theta):
+        W1_, b1_, w2_, b2_ = theta[:hidden * d].reshape(hidden, d), theta[hidden * d:hidden * d + hidden], \
+            theta[hidden * d + hidden:hidden * d + 2 * hidden], theta[-1]
+        return O.bce_mean(O.score_mlp(x, W1_, b1_, w2_, b2_), z)
+
+    theta0 = np.concatenate([W1.reshape(-1), b1, w2, [b2]]).astype(np.float64)
+    probe = theta0.copy()
+    g_fd = _fd(lambda: objective(probe), probe)
+    lr = 1e-3
+    out = O.assistant_step_mlp(x, f, W1, W1_bits, b1, w2, b2, lr, T=T)
+    theta1 = np.concatenate([out["W1"].reshape(-1), out["b1"], out["w2"], [out["b2"]]]).astype(np.float64)
+    # the update is -lr times the finite-difference gradient (fp32 rounding of the parameters aside)
+    assert np.allclose(theta0 - theta1, lr * g_fd, rtol=2e-3, atol=2e-7)
+    drop = objective(theta0) - objective(theta1)
+    assert drop > 0 and abs(drop - lr * float(g_fd @ g_fd)) <= 0.02 * lr * float(g_fd @ g_fd)
+    assert np.array_equal(out["W1_bf16"], O.round_bf16(out["W1"]))
+    assert np.array_equal(out["z"], z)
