@@ -164,6 +164,30 @@ aa_status aa_shrink_compact(aa_ctx* ctx, const float* score, int64_t n, int64_t 
                             int32_t* out_idx, int64_t capacity, int32_t* out_count, uint8_t* out_mask);
 
 /*
+ * Batch cut + cursor: the batch Algorithm 1 (Assistant.sample_batch) returns, cut out of the ordered
+ * survivor list of a screened pool.  Algorithm 1 stops as soon as the batch holds batch_size
+ * instances, so its batch is the first batch_size entries of the list and its walk over the
+ * (shuffled) candidate list ends right after the last one taken; the next call starts there.
+ * For sequence tasks (Sec. 6.2: batches of a given number of tokens) the batch is the longest prefix
+ * of the list whose sentence lengths add up to at most token_budget.
+ *   idx, count_dev : out_idx / out_count of aa_score_shrink (candidate k = stored row k, i.e. no
+ *                    candidate list); idx_capacity bounds the device count.  n_cand = pool size.
+ *   batch_size     : most instances in the batch (0 = no limit).
+ *   lengths        : nullable; lengths[r] = tokens of stored row r (n_stored rows, negative counts
+ *                    as 0); with it token_budget applies.  A list entry outside the rows latches
+ *                    AA_ERR_BAD_INDEX and counts as length 0.
+ *   out_m[0]       : instances in the batch, b.
+ *   out_consumed[0]: candidates the walk covered: idx[b-1] + 1 when a limit ended it (0 if not even
+ *                    the first survivor fits), n_cand when the survivors ran out first.
+ *   out_offsets    : nullable (needs lengths), offsets_capacity entries: out_offsets[k] = tokens of
+ *                    the first k batch instances, k = 0..b — the offsets aa_instance_loss takes.
+ * All outputs are device memory; nothing is read back.
+ */
+aa_status aa_batch_cut(aa_ctx* ctx, const int32_t* idx, const int32_t* count_dev, int64_t idx_capacity, int64_t n_cand,
+                       int64_t batch_size, const int32_t* lengths, int64_t n_stored, int64_t token_budget,
+                       int32_t* out_m, int32_t* out_consumed, int32_t* out_offsets, int64_t offsets_capacity);
+
+/*
  * aa_shrink_compact for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this is a deployment variant of the entry point above.)
  *

@@ -318,3 +318,28 @@ def assistant_step_mlp(x, f, W1, W1_bf16, b1, w2, b2, lr, T=None, row_idx=None):
         "W1": W1_new, "W1_bf16": round_bf16(W1_new), "b1": sgd(b1, gb1, lr), "w2": sgd(w2, gw2, lr),
         "b2": sgd(np.array([b2], np.float32), np.array([gb2]), lr)[0], "z": z, "grads": (gW1, gb1, gw2, gb2), "a": a, "s": s,
     }
+
+
+def batch_cut(B, n_cand: int, batch_size: int = 0, lengths=None, token_budget: int = 0):
+    """The batch Algorithm 1 returns, cut from the ordered survivors B, written as the literal walk: take survivors in
+    order until the batch holds batch_size of them (0 = no limit) or, with sentence lengths, until the next one would
+    push the token total past token_budget.  Returns (b, consumed, offsets): consumed = position right after the last
+    instance taken when a limit ended the walk, n_cand when the survivors ran out; offsets = running token totals."""
+    B = np.asarray(B, dtype=np.int64)
+    b, tokens, offsets, limited = 0, 0, [0], False
+    for r in B:
+        if batch_size > 0 and b == batch_size:
+            limited = True
+            break
+        if lengths is not None:
+            ln = max(int(lengths[r]), 0)
+            if tokens + ln > token_budget:
+                limited = True
+                break
+            tokens += ln
+            offsets.append(tokens)
+        b += 1
+    if batch_size > 0 and b == batch_size:
+        limited = True
+    consumed = (int(B[b - 1]) + 1 if b > 0 else 0) if limited else int(n_cand)
+    return b, consumed, np.asarray(offsets, dtype=np.int64)

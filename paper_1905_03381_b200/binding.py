@@ -26,7 +26,7 @@ AA_THRESH_VALUE, AA_THRESH_BATCH_MEAN = 0, 1
 EXPORTS = (
     "aa_status_string", "aa_workspace_bytes", "aa_create", "aa_destroy", "aa_score_shrink",
     "aa_shrink_compact", "aa_instance_loss", "aa_assistant_step", "aa_step_host_staging_bytes", "aa_step_host",
-    "aa_device_status", "aa_launch_count", "aa_shrink_compact_static",
+    "aa_device_status", "aa_launch_count", "aa_shrink_compact_static", "aa_batch_cut",
 )
 AA_STATIC_MAX_CANDIDATES = 1 << 22
 
@@ -85,6 +85,8 @@ def lib() -> ctypes.CDLL:
                                         c_void_p, c_int64, c_void_p, c_void_p]
         L.aa_shrink_compact_static.argtypes = [c_void_p, c_int64, c_int64, c_float, c_uint64, c_uint64,
                                                c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_void_p]
+        L.aa_batch_cut.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_int64, c_int64,
+                                   c_void_p, c_void_p, c_void_p, c_int64]
         L.aa_instance_loss.argtypes = [c_void_p, POINTER(aa_logits), c_void_p, c_void_p, c_int64, c_void_p, c_void_p]
         L.aa_assistant_step.argtypes = [c_void_p, POINTER(aa_feat), c_void_p, c_void_p, POINTER(aa_assistant),
                                         c_float, c_int32, c_float]
@@ -248,6 +250,17 @@ class AutoAssist:
         self._ok(self._L.aa_shrink_compact(self._ctx, score.data_ptr(), score.numel() if n is None else n, id_base,
                                            mix, seed, step, out_idx.data_ptr(), out_idx.numel(),
                                            out_count.data_ptr(), _ptr(out_mask)), "aa_shrink_compact")
+
+    def aa_batch_cut(self, idx: torch.Tensor, count_dev: torch.Tensor, n_cand: int, out_m: torch.Tensor,
+                     out_consumed: torch.Tensor, batch_size: int = 0, lengths=None, token_budget: int = 0, out_offsets=None):
+        """The batch Algorithm 1 returns (first batch_size survivors, or the longest prefix within a token budget) and
+        how many candidates its walk covered; all results stay on the device."""
+        _check(lengths, torch.int32, "lengths")
+        _check(out_offsets, torch.int32, "out_offsets")
+        self._ok(self._L.aa_batch_cut(self._ctx, idx.data_ptr(), _ptr(count_dev), idx.numel(), n_cand, batch_size,
+                                      _ptr(lengths), 0 if lengths is None else lengths.numel(), token_budget,
+                                      out_m.data_ptr(), out_consumed.data_ptr(), _ptr(out_offsets),
+                                      0 if out_offsets is None else out_offsets.numel()), "aa_batch_cut")
 
     def aa_instance_loss(self, logits: aa_logits, labels: torch.Tensor, out_loss: torch.Tensor, offsets=None,
                          n_seg=None, count_dev=None):

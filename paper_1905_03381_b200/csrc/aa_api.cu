@@ -251,6 +251,18 @@ aa_status aa_shrink_compact(aa_ctx* ctx, const float* score, int64_t n, int64_t 
     return launch_shrink_from_scores(c, score, sp);
 }
 
+aa_status aa_batch_cut(aa_ctx* ctx, const int32_t* idx, const int32_t* count_dev, int64_t idx_capacity, int64_t n_cand,
+                       int64_t batch_size, const int32_t* lengths, int64_t n_stored, int64_t token_budget, int32_t* out_m,
+                       int32_t* out_consumed, int32_t* out_offsets, int64_t offsets_capacity) {
+    if (!ctx || !out_m || !out_consumed || idx_capacity < 0 || n_cand < 0 || n_cand > 0x7FFFFFFFll || batch_size < 0)
+        return AA_ERR_INVALID_ARG;
+    if (idx_capacity > 0 && !idx) return AA_ERR_INVALID_ARG;
+    if (lengths && (token_budget < 0 || n_stored < 0)) return AA_ERR_INVALID_ARG;
+    if (out_offsets && (!lengths || offsets_capacity < 1)) return AA_ERR_INVALID_ARG;
+    return launch_batch_cut(&ctx->impl, idx, count_dev, idx_capacity, n_cand, n_stored, batch_size, lengths, token_budget, out_m,
+                            out_consumed, out_offsets, offsets_capacity);
+}
+
 aa_status aa_instance_loss(aa_ctx* ctx, const aa_logits* lg, const int32_t* labels, const int32_t* offsets, int64_t n_seg,
                            const int32_t* count_dev, float* out_loss) {
     if (!ctx || !lg || lg->rows < 0 || lg->cols <= 0 || lg->row_stride < lg->cols) return AA_ERR_INVALID_ARG;

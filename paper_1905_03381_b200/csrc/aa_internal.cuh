@@ -224,6 +224,10 @@ aa_status launch_shrink_from_scores(aa_ctx_impl* c, const float* score, ShrinkPa
 struct LossParams;
 aa_status launch_instance_loss_tma(aa_ctx_impl* c, const LossParams& p, int dtype);
 
+aa_status launch_batch_cut(aa_ctx_impl* c, const int32_t* idx, const int32_t* count_dev, int64_t m_host, int64_t n_cand,
+                           int64_t n_stored, int64_t batch_size, const int32_t* lengths, int64_t token_budget, int32_t* out_m,
+                           int32_t* out_consumed, int32_t* out_offsets, int64_t offsets_capacity);
+
 aa_status launch_instance_loss(aa_ctx_impl* c, const aa_logits& lg, const int32_t* labels, const int32_t* offsets,
                                int64_t n_seg, const int32_t* count_dev, float* out_loss);
 

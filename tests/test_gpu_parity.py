@@ -221,6 +221,45 @@ def test_csr_screen(aa, n, d, max_len):
     check_screen(gpu, s, O.shrink(g, 0.2, 4, 8), O.accept_prob(g, 0.2), c, None, float(np.linalg.norm(wh)), scale)
 
 
+def test_batch_cut_and_cursor(aa):
+    """aa_batch_cut against the oracle's literal walk: integer work, bit-exact."""
+    n = 70001
+    s = W.normal((n,), 1.5, 77, torch.float32, DEV)
+    idx = torch.full((n,), -7, dtype=torch.int32, device=DEV)
+    cnt = torch.zeros(1, dtype=torch.int32, device=DEV)
+    aa.aa_shrink_compact(s, 0.2, 5, 6, idx, cnt)
+    torch.cuda.synchronize()
+    m = int(cnt.item())
+    Bfull = idx.cpu().numpy()[:m]
+    lengths = W.randint(8, 129, (n,), 78, DEV)
+    lengths[int(Bfull[3])] = -4                                   # a negative count is a zero-length sentence
+    lh = lengths.cpu().numpy()
+    out_m = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out_c = torch.zeros(1, dtype=torch.int32, device=DEV)
+    off = torch.full((m + 1,), -7, dtype=torch.int32, device=DEV)
+    cases = [dict(batch_size=1), dict(batch_size=1000), dict(batch_size=m), dict(batch_size=m + 5), dict(),
+             dict(lengths=lengths, token_budget=25000), dict(lengths=lengths, token_budget=25000, batch_size=100),
+             dict(lengths=lengths, token_budget=3), dict(lengths=lengths, token_budget=10 ** 8),
+             dict(lengths=lengths, token_budget=2 * 10 ** 6)]     # several scan chunks with a carry
+    for kw in cases:
+        off.fill_(-7)
+        use_off = "lengths" in kw
+        aa.aa_batch_cut(idx, cnt, n, out_m, out_c, out_offsets=off if use_off else None, **kw)
+        torch.cuda.synchronize()
+        b_ref, c_ref, off_ref = O.batch_cut(Bfull, n, batch_size=kw.get("batch_size", 0), lengths=lh if use_off else None,
+                                            token_budget=kw.get("token_budget", 0))
+        assert (int(out_m.item()), int(out_c.item())) == (b_ref, c_ref), kw
+        if use_off:
+            got = off.cpu().numpy()
+            assert np.array_equal(got[:b_ref + 1], off_ref) and np.all(got[b_ref + 1:] == -7)
+    # an empty survivor list consumes the whole pool
+    zero = torch.zeros(1, dtype=torch.int32, device=DEV)
+    aa.aa_batch_cut(idx, zero, n, out_m, out_c, batch_size=10)
+    torch.cuda.synchronize()
+    assert (int(out_m.item()), int(out_c.item())) == (0, n)
+    assert aa.aa_device_status() == B.AA_OK
+
+
 # --------------------------------------------------------------------------
 # per-instance loss
 # --------------------------------------------------------------------------

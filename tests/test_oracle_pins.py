@@ -501,3 +501,29 @@ def test_composed_mlp_step_descends_the_objective_to_first_order():
     assert drop > 0 and abs(drop - lr * float(g_fd @ g_fd)) <= 0.02 * lr * float(g_fd @ g_fd)
     assert np.array_equal(out["W1_bf16"], O.round_bf16(out["W1"]))
     assert np.array_equal(out["z"], z)
+
+
+def test_batch_cut_is_the_literal_walk_of_algorithm_1():
+    """batch_cut on the ordered survivors equals the sequential Algorithm 1 loop (batch and candidates consumed), and the
+    token-budget form has the closed forms of unit lengths and of a budget nothing fits in."""
+    rng = np.random.default_rng(9)
+    n = 5000
+    g = rng.uniform(0.05, 0.95, n)
+    keep = O.shrink(g, 0.1, 4, 2)
+    Bfull = O.compact(keep)
+    for bs in (1, 7, 64, len(Bfull), len(Bfull) + 10):
+        Bseq, consumed_seq = O.sample_batch(g, 0.1, 4, 2, bs)
+        b, consumed, _ = O.batch_cut(Bfull, n, batch_size=bs)
+        assert b == len(Bseq) and np.array_equal(Bfull[:b], Bseq) and consumed == consumed_seq
+    ones = np.ones(n, np.int32)
+    b, consumed, off = O.batch_cut(Bfull, n, lengths=ones, token_budget=100)
+    assert b == 100 and consumed == Bfull[99] + 1 and np.array_equal(off, np.arange(101))
+    b, consumed, off = O.batch_cut(Bfull, n, lengths=ones * 5, token_budget=4)
+    assert (b, consumed, list(off)) == (0, 0, [0])
+    b, consumed, off = O.batch_cut(Bfull, n, lengths=ones, token_budget=10 ** 9)
+    assert b == len(Bfull) and consumed == n and off[-1] == len(Bfull)
+    lengths = rng.integers(8, 129, n).astype(np.int32)
+    b, consumed, off = O.batch_cut(Bfull, n, lengths=lengths, token_budget=25000, batch_size=300)
+    assert b == 300 and off[-1] == lengths[Bfull[:300]].sum() <= 25000      # the instance limit binds first here
+    b, consumed, off = O.batch_cut(Bfull, n, lengths=lengths, token_budget=2500)
+    assert off[-1] <= 2500 < off[-1] + lengths[Bfull[b]] and np.array_equal(np.diff(off), lengths[Bfull[:b]])
