@@ -164,6 +164,19 @@ aa_status aa_shrink_compact(aa_ctx* ctx, const float* score, int64_t n, int64_t 
                             int32_t* out_idx, int64_t capacity, int32_t* out_count, uint8_t* out_mask);
 
 /*
+ * Hard shrinking (Sec. 4.2, Eq. "shrinking_grad"; the SK method of Sec. 4.4): an instance is used
+ * only if its objective value or gradient magnitude is at least T.  value[i] is that quantity for
+ * instance i (e.g. the losses of aa_instance_loss); out_idx receives the ascending list of i with
+ * value[i] >= threshold, out_count its length, out_mask (nullable) one byte per instance.  No random
+ * draw is involved; NaN values are dropped.  Capacity overflow latches AA_ERR_CAPACITY as in
+ * aa_score_shrink.  aa_sk_threshold gives the schedule T_k = G / k of the convergence theorem
+ * (Sec. 5, Theorem 1) for step k >= 1 (HOST helper).
+ */
+aa_status aa_threshold_compact(aa_ctx* ctx, const float* value, int64_t n, float threshold,
+                               int32_t* out_idx, int64_t capacity, int32_t* out_count, uint8_t* out_mask);
+float aa_sk_threshold(float G, int64_t k);
+
+/*
  * Batch cut + cursor: the batch Algorithm 1 (Assistant.sample_batch) returns, cut out of the ordered
  * survivor list of a screened pool.  Algorithm 1 stops as soon as the batch holds batch_size
  * instances, so its batch is the first batch_size entries of the list and its walk over the

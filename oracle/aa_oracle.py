@@ -343,3 +343,17 @@ def batch_cut(B, n_cand: int, batch_size: int = 0, lengths=None, token_budget: i
         limited = True
     consumed = (int(B[b - 1]) + 1 if b > 0 else 0) if limited else int(n_cand)
     return b, consumed, np.asarray(offsets, dtype=np.int64)
+
+
+def hard_shrink(value, T: float) -> np.ndarray:
+    """Hard shrinking (Eq. "shrinking_grad"): instance i is used iff its objective value / gradient magnitude is >= T."""
+    value = np.asarray(value, dtype=np.float32)
+    keep = np.zeros(value.size, dtype=np.uint8)
+    for i in range(value.size):
+        keep[i] = 1 if float(value[i]) >= float(np.float32(T)) else 0
+    return keep
+
+
+def sk_threshold(G: float, k: int) -> float:
+    """Threshold schedule of the convergence theorem: T_k = G / k."""
+    return float(np.float32(G) / np.float32(k))

@@ -26,7 +26,7 @@ AA_THRESH_VALUE, AA_THRESH_BATCH_MEAN = 0, 1
 EXPORTS = (
     "aa_status_string", "aa_workspace_bytes", "aa_create", "aa_destroy", "aa_score_shrink",
     "aa_shrink_compact", "aa_instance_loss", "aa_assistant_step", "aa_step_host_staging_bytes", "aa_step_host",
-    "aa_device_status", "aa_launch_count", "aa_shrink_compact_static", "aa_batch_cut",
+    "aa_device_status", "aa_launch_count", "aa_shrink_compact_static", "aa_batch_cut", "aa_threshold_compact", "aa_sk_threshold",
 )
 AA_STATIC_MAX_CANDIDATES = 1 << 22
 
@@ -85,6 +85,9 @@ def lib() -> ctypes.CDLL:
                                         c_void_p, c_int64, c_void_p, c_void_p]
         L.aa_shrink_compact_static.argtypes = [c_void_p, c_int64, c_int64, c_float, c_uint64, c_uint64,
                                                c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_void_p]
+        L.aa_threshold_compact.argtypes = [c_void_p, c_void_p, c_int64, c_float, c_void_p, c_int64, c_void_p, c_void_p]
+        L.aa_sk_threshold.restype = c_float
+        L.aa_sk_threshold.argtypes = [c_float, c_int64]
         L.aa_batch_cut.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_int64, c_int64,
                                    c_void_p, c_void_p, c_void_p, c_int64]
         L.aa_instance_loss.argtypes = [c_void_p, POINTER(aa_logits), c_void_p, c_void_p, c_int64, c_void_p, c_void_p]
@@ -118,6 +121,11 @@ def aa_shrink_compact_static(score: torch.Tensor, mix: float, seed: int, step: i
                                             _ptr(out_mask), _ptr(out_status), s.cuda_stream)
     if st != AA_OK:
         raise AutoAssistError(st, "aa_shrink_compact_static")
+
+
+def aa_sk_threshold(G: float, k: int) -> float:
+    """T_k = G / k, the shrinking threshold schedule of the paper's convergence theorem."""
+    return float(lib().aa_sk_threshold(G, k))
 
 
 def _ptr(t):
@@ -250,6 +258,14 @@ class AutoAssist:
         self._ok(self._L.aa_shrink_compact(self._ctx, score.data_ptr(), score.numel() if n is None else n, id_base,
                                            mix, seed, step, out_idx.data_ptr(), out_idx.numel(),
                                            out_count.data_ptr(), _ptr(out_mask)), "aa_shrink_compact")
+
+    def aa_threshold_compact(self, value: torch.Tensor, threshold: float, out_idx: torch.Tensor, out_count: torch.Tensor,
+                             out_mask=None, n=None):
+        """Hard shrinking: ordered list of the instances whose value (loss or gradient magnitude) is >= threshold."""
+        _check(value, torch.float32, "value")
+        self._ok(self._L.aa_threshold_compact(self._ctx, value.data_ptr(), value.numel() if n is None else n, threshold,
+                                              out_idx.data_ptr(), out_idx.numel(), out_count.data_ptr(), _ptr(out_mask)),
+                 "aa_threshold_compact")
 
     def aa_batch_cut(self, idx: torch.Tensor, count_dev: torch.Tensor, n_cand: int, out_m: torch.Tensor,
                      out_consumed: torch.Tensor, batch_size: int = 0, lengths=None, token_budget: int = 0, out_offsets=None):

@@ -251,6 +251,20 @@ aa_status aa_shrink_compact(aa_ctx* ctx, const float* score, int64_t n, int64_t 
     return launch_shrink_from_scores(c, score, sp);
 }
 
+aa_status aa_threshold_compact(aa_ctx* ctx, const float* value, int64_t n, float threshold, int32_t* out_idx, int64_t capacity,
+                               int32_t* out_count, uint8_t* out_mask) {
+    if (!ctx || (n > 0 && !value) || threshold != threshold) return AA_ERR_INVALID_ARG;
+    aa_ctx_impl* c = &ctx->impl;
+    ShrinkParams sp;
+    aa_status st = base_shrink_params(sp, n, n, nullptr, 0, 0.0f, 0, 0, out_idx, capacity, out_count, nullptr, out_mask);
+    if (st != AA_OK) return st;
+    sp.hard = 1;
+    sp.hard_threshold = threshold;
+    if (n > c->max_rows) return AA_ERR_WORKSPACE;
+    if (n == 0) return cuda_ok(cudaMemsetAsync(out_count, 0, sizeof(int32_t), c->stream));
+    return launch_shrink_from_scores(c, value, sp);
+}
+
 aa_status aa_batch_cut(aa_ctx* ctx, const int32_t* idx, const int32_t* count_dev, int64_t idx_capacity, int64_t n_cand,
                        int64_t batch_size, const int32_t* lengths, int64_t n_stored, int64_t token_budget, int32_t* out_m,
                        int32_t* out_consumed, int32_t* out_offsets, int64_t offsets_capacity) {
@@ -413,6 +427,8 @@ aa_status aa_device_status(aa_ctx* ctx, int32_t* latched) {
     }
     return AA_OK;
 }
+
+float aa_sk_threshold(float G, int64_t k) { return k >= 1 ? G / (float)k : G; }
 
 int64_t aa_launch_count(const aa_ctx* ctx) { return ctx ? ctx->impl.launches : -1; }
 

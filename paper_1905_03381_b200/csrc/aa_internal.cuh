@@ -55,6 +55,8 @@ struct ShrinkParams {
     const int32_t* row_idx;  // optional candidate list
     int64_t id_base;
     float mix;               // gamma of Algorithm 1
+    int hard;                // 1: keep iff value >= hard_threshold (hard shrinking, no random draw)
+    float hard_threshold;
     uint32_t seed_lo, seed_hi, step_lo, step_hi;
     int32_t* out_idx;
     int64_t capacity;

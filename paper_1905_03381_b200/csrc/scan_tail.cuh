@@ -33,12 +33,14 @@ __device__ __forceinline__ long long candidate_row(const ShrinkParams& p, long l
 
 // Keep/skip for candidate k with pre-activation s:  c < gamma + (1 - gamma) sigmoid(s),
 // c drawn from Philox at counter (instance id, step).  Unreadable rows are skipped.
+// In hard mode s is the instance's loss or gradient magnitude and the decision is s >= T.
 __device__ __forceinline__ bool keep_decision(const ShrinkParams& p, long long k, float s) {
     long long r = k;
     if (p.row_idx) {
         r = p.row_idx[k];
         if ((unsigned long long)r >= (unsigned long long)p.n_stored) return false;
     }
+    if (p.hard) return s >= p.hard_threshold;   // hard shrinking (Eq. "shrinking_grad"); NaN compares false
     const float prob = fmaf(1.0f - p.mix, sigmoid_f32(s), p.mix);
     const float c = philox_uniform(p, (uint64_t)(p.id_base + r));
     return c < prob;

@@ -221,6 +221,25 @@ def test_csr_screen(aa, n, d, max_len):
     check_screen(gpu, s, O.shrink(g, 0.2, 4, 8), O.accept_prob(g, 0.2), c, None, float(np.linalg.norm(wh)), scale)
 
 
+def test_hard_threshold_shrinking(aa):
+    """aa_threshold_compact against the oracle: comparisons of fp32 values, bit-exact."""
+    for n, T in ((1, 0.5), (1023, 0.0), (70001, 1.0), (70001, 50.0), (120000, float(B.aa_sk_threshold(6.0, 4)))):
+        v = (W.normal((n,), 1.0, 80 + n, torch.float32, DEV).abs() * 1.5).contiguous()
+        if n > 10:
+            v[3] = float("nan"); v[4] = T; v[5] = float("inf")
+        idx = torch.full((n,), -7, dtype=torch.int32, device=DEV)
+        cnt = torch.zeros(1, dtype=torch.int32, device=DEV)
+        mask = torch.full((n,), 9, dtype=torch.uint8, device=DEV)
+        aa.aa_threshold_compact(v, T, idx, cnt, mask)
+        torch.cuda.synchronize()
+        keep = O.hard_shrink(v.cpu().numpy(), T)
+        m = int(cnt.item())
+        assert np.array_equal(mask.cpu().numpy(), keep)
+        assert m == int(keep.sum()) and np.array_equal(idx.cpu().numpy()[:m], O.compact(keep)) and bool((idx[m:] == -7).all())
+    assert B.aa_sk_threshold(6.0, 4) == O.sk_threshold(6.0, 4) == 1.5
+    assert aa.aa_device_status() == B.AA_OK
+
+
 def test_batch_cut_and_cursor(aa):
     """aa_batch_cut against the oracle's literal walk: integer work, bit-exact."""
     n = 70001

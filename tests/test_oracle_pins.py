@@ -527,3 +527,16 @@ def test_batch_cut_is_the_literal_walk_of_algorithm_1():
     assert b == 300 and off[-1] == lengths[Bfull[:300]].sum() <= 25000      # the instance limit binds first here
     b, consumed, off = O.batch_cut(Bfull, n, lengths=lengths, token_budget=2500)
     assert off[-1] <= 2500 < off[-1] + lengths[Bfull[b]] and np.array_equal(np.diff(off), lengths[Bfull[:b]])
+
+
+def test_hard_shrinking_rule():
+    v = np.array([0.0, 0.5, 0.5000001, 0.4999999, np.nan, np.inf, -1.0, 2.0], np.float32)
+    keep = O.hard_shrink(v, 0.5)
+    assert list(keep) == [0, 1, 1, 0, 0, 1, 0, 1]                  # >= keeps, NaN drops
+    rng = np.random.default_rng(3)
+    v = rng.exponential(1.0, 20000).astype(np.float32)
+    counts = [int(O.hard_shrink(v, T).sum()) for T in (0.0, 0.5, 1.0, 2.0, 50.0)]
+    assert counts[0] == v.size and counts[-1] == 0 and all(a >= b for a, b in zip(counts, counts[1:]))
+    assert abs(counts[2] / v.size - math.exp(-1.0)) < 0.01          # P(Exp(1) >= 1) = 1/e
+    assert np.array_equal(O.compact(O.hard_shrink(v, 1.0)), np.nonzero(v >= np.float32(1.0))[0])
+    assert O.sk_threshold(3.0, 1) == 3.0 and math.isclose(O.sk_threshold(3.0, 12), 0.25, rel_tol=1e-6)
