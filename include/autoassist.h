@@ -261,6 +261,27 @@ aa_status aa_assistant_step(aa_ctx* ctx, const aa_feat* feat, const float* loss,
                             aa_assistant* assistant, float lr, int32_t thresh_mode, float threshold);
 
 /*
+ * Step 5 with Adam in place of SGD (the paper trained its Assistants with Adam, Sec. 6.1).  Labels and gradient exactly as
+ * in aa_assistant_step; the update of every parameter p with mean gradient g is
+ *   m <- beta1 m + (1 - beta1) g,   v <- beta2 v + (1 - beta2) g^2,
+ *   p <- p - lr (m / (1 - beta1^t)) / (sqrt(v / (1 - beta2^t)) + eps),      t = state->t + 1,
+ * in fp32.  state (HOST struct) is caller-owned: m and v are DEVICE arrays laid out like the flattened parameters
+ * (linear: w[d] then b, d + 1 floats; two-layer: W1[hidden*d], b1[hidden], w2[hidden], b2, hidden*(d+2) + 1 floats),
+ * zero before the first step; the call advances state->t.  A batch that turns out empty on the device leaves parameters
+ * and moments unchanged (t still advances).  With CSR features every weight is updated, not only the batch's columns:
+ * a first moment keeps moving its weight while it decays.
+ */
+typedef struct {
+    float beta1, beta2, eps;
+    int32_t reserved;
+    int64_t t;               /* steps taken so far */
+    float* m;
+    float* v;
+} aa_adam;
+aa_status aa_assistant_step_adam(aa_ctx* ctx, const aa_feat* feat, const float* loss, const int32_t* count_dev,
+                                 aa_assistant* assistant, aa_adam* state, float lr, int32_t thresh_mode, float threshold);
+
+/*
  * One whole step for callers whose data lives in HOST memory (pinned memory for full copy speed):
  * copies the candidate features, the Boss logits and the labels to the device staging buffer,
  * runs steps 1-5 above (dense linear Assistant), copies the batch list, its count, the

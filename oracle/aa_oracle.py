@@ -357,3 +357,21 @@ def hard_shrink(value, T: float) -> np.ndarray:
 def sk_threshold(G: float, k: int) -> float:
     """Threshold schedule of the convergence theorem: T_k = G / k."""
     return float(np.float32(G) / np.float32(k))
+
+
+def adam(param, m, v, grad, lr: float, beta1: float, beta2: float, eps: float, t: int):
+    """One Adam update (Kingma & Ba; the optimizer the paper's Assistants were trained with), elementwise in fp64 on
+    fp32 state: returns (param, m, v) rounded once to fp32.  t = number of this step, starting at 1."""
+    p64 = np.asarray(param, np.float32).astype(np.float64)
+    m64 = np.asarray(m, np.float32).astype(np.float64)
+    v64 = np.asarray(v, np.float32).astype(np.float64)
+    g64 = np.asarray(grad, np.float64).reshape(p64.shape)
+    b1, b2 = float(np.float32(beta1)), float(np.float32(beta2))
+    m_new = np.empty_like(m64); v_new = np.empty_like(v64); p_new = np.empty_like(p64)
+    for j in np.ndindex(p64.shape):
+        m_new[j] = b1 * m64[j] + (1.0 - b1) * g64[j]
+        v_new[j] = b2 * v64[j] + (1.0 - b2) * g64[j] * g64[j]
+        m_hat = m_new[j] / (1.0 - b1 ** t)
+        v_hat = v_new[j] / (1.0 - b2 ** t)
+        p_new[j] = p64[j] - lr * m_hat / (np.sqrt(v_hat) + float(np.float32(eps)))
+    return p_new.astype(np.float32), m_new.astype(np.float32), v_new.astype(np.float32)

@@ -26,7 +26,7 @@ AA_THRESH_VALUE, AA_THRESH_BATCH_MEAN = 0, 1
 EXPORTS = (
     "aa_status_string", "aa_workspace_bytes", "aa_create", "aa_destroy", "aa_score_shrink",
     "aa_shrink_compact", "aa_instance_loss", "aa_assistant_step", "aa_step_host_staging_bytes", "aa_step_host",
-    "aa_device_status", "aa_launch_count", "aa_shrink_compact_static", "aa_batch_cut", "aa_threshold_compact", "aa_sk_threshold",
+    "aa_device_status", "aa_launch_count", "aa_shrink_compact_static", "aa_batch_cut", "aa_threshold_compact", "aa_sk_threshold", "aa_assistant_step_adam",
 )
 AA_STATIC_MAX_CANDIDATES = 1 << 22
 
@@ -53,6 +53,22 @@ class aa_logits(Structure):
         ("data", c_void_p), ("dtype", c_int32), ("reserved", c_int32),
         ("rows", c_int64), ("cols", c_int64), ("row_stride", c_int64),
     ]
+
+
+class aa_adam(Structure):
+    _fields_ = [("beta1", c_float), ("beta2", c_float), ("eps", c_float), ("reserved", c_int32), ("t", c_int64),
+                ("m", c_void_p), ("v", c_void_p)]
+
+
+def adam_state(m: torch.Tensor, v: torch.Tensor, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8) -> aa_adam:
+    """Adam moments (fp32 device tensors laid out like the flattened parameters, zero before the first step)."""
+    _check(m, torch.float32, "m")
+    _check(v, torch.float32, "v")
+    st = aa_adam()
+    st.beta1, st.beta2, st.eps, st.t = beta1, beta2, eps, 0
+    st.m, st.v = m.data_ptr(), v.data_ptr()
+    st._keep = (m, v)
+    return st
 
 
 class AutoAssistError(RuntimeError):
@@ -85,6 +101,8 @@ def lib() -> ctypes.CDLL:
                                         c_void_p, c_int64, c_void_p, c_void_p]
         L.aa_shrink_compact_static.argtypes = [c_void_p, c_int64, c_int64, c_float, c_uint64, c_uint64,
                                                c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_void_p]
+        L.aa_assistant_step_adam.argtypes = [c_void_p, POINTER(aa_feat), c_void_p, c_void_p, POINTER(aa_assistant),
+                                             POINTER(aa_adam), c_float, c_int32, c_float]
         L.aa_threshold_compact.argtypes = [c_void_p, c_void_p, c_int64, c_float, c_void_p, c_int64, c_void_p, c_void_p]
         L.aa_sk_threshold.restype = c_float
         L.aa_sk_threshold.argtypes = [c_float, c_int64]
@@ -292,6 +310,14 @@ class AutoAssist:
         mode = AA_THRESH_BATCH_MEAN if threshold is None else AA_THRESH_VALUE
         self._ok(self._L.aa_assistant_step(self._ctx, byref(feat), loss.data_ptr(), _ptr(count_dev), byref(assistant),
                                            lr, mode, 0.0 if threshold is None else threshold), "aa_assistant_step")
+
+    def aa_assistant_step_adam(self, feat: aa_feat, loss: torch.Tensor, assistant: aa_assistant, state: aa_adam, lr: float,
+                               threshold=None, count_dev=None):
+        """aa_assistant_step with Adam; state.t advances."""
+        mode = AA_THRESH_BATCH_MEAN if threshold is None else AA_THRESH_VALUE
+        self._ok(self._L.aa_assistant_step_adam(self._ctx, byref(feat), loss.data_ptr(), _ptr(count_dev), byref(assistant),
+                                                byref(state), lr, mode, 0.0 if threshold is None else threshold),
+                 "aa_assistant_step_adam")
 
     def host_step_plan(self, x_host: torch.Tensor, logits_host: torch.Tensor):
         """Descriptors and a device staging buffer for aa_step_host on HOST tensors of these shapes."""

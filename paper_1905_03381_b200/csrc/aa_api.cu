@@ -2,6 +2,7 @@
 // Every entry point validates on the host, then enqueues kernels on the context's stream.
 #include <new>
 #include <stdio.h>
+#include <math.h>
 #include <string.h>
 
 #include "aa_internal.cuh"
@@ -317,6 +318,28 @@ aa_status aa_assistant_step(aa_ctx* ctx, const aa_feat* feat, const float* loss,
     f.mean_nnz = (feat->nnz > 0 && feat->n > 0) ? (float)feat->nnz / (float)feat->n : 32.0f;
     return launch_assistant_step_csr(c, f, feat->row_idx, feat->n, m_host, count_dev, loss, a->w, a->b, lr, thresh_mode,
                                      threshold);
+}
+
+aa_status aa_assistant_step_adam(aa_ctx* ctx, const aa_feat* feat, const float* loss, const int32_t* count_dev, aa_assistant* a,
+                                 aa_adam* state, float lr, int32_t thresh_mode, float threshold) {
+    if (!ctx || !state || !state->m || !state->v || state->t < 0) return AA_ERR_INVALID_ARG;
+    if (!(state->beta1 >= 0.0f && state->beta1 < 1.0f) || !(state->beta2 >= 0.0f && state->beta2 < 1.0f) || !(state->eps >= 0.0f))
+        return AA_ERR_INVALID_ARG;
+    const double t = (double)(state->t + 1);
+    AdamArgs args;
+    args.on = 1;
+    args.beta1 = state->beta1;
+    args.beta2 = state->beta2;
+    args.eps = state->eps;
+    args.corr1 = (float)(1.0 / (1.0 - pow((double)state->beta1, t)));
+    args.corr2 = (float)(1.0 / (1.0 - pow((double)state->beta2, t)));
+    args.m = state->m;
+    args.v = state->v;
+    ctx->impl.adam = args;
+    const aa_status st = aa_assistant_step(ctx, feat, loss, count_dev, a, lr, thresh_mode, threshold);
+    ctx->impl.adam.on = 0;
+    if (st == AA_OK) state->t += 1;
+    return st;
 }
 
 namespace {

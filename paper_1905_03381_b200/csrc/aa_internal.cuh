@@ -24,6 +24,16 @@ constexpr int kScanThreads = 128;      // CTA size of the score/shrink/compact k
 constexpr int kMaxParts = 1024;        // upper bound on per-CTA gradient partials
 constexpr unsigned kSpinLimit = 1u << 22;   // polls before a look-back wait gives up
 
+// Optimizer of the Assistant update: plain SGD, or Adam with caller-owned moment arrays laid out like the
+// flattened parameters (linear: w[d] then b; two-layer: W1[hidden*d], b1[hidden], w2[hidden], b2).
+struct AdamArgs {
+    int on;
+    float beta1, beta2, eps;
+    float corr1, corr2;      // 1 / (1 - beta1^t), 1 / (1 - beta2^t) for this step
+    float* m;
+    float* v;
+};
+
 struct aa_ctx_impl {
     char* ws;
     size_t ws_bytes;
@@ -37,6 +47,7 @@ struct aa_ctx_impl {
     float* row_scratch;               // max_rows floats: row losses / residuals
     float* partials;                  // gradient partial sums
     int64_t partial_floats;
+    AdamArgs adam;                    // optimizer of the step being enqueued (on = 0: SGD)
     int64_t launches;
     uint64_t scans_since_clear;
     // two-layer Assistant step (present when the context was sized with max_hidden > 0)
@@ -69,6 +80,16 @@ struct ShrinkParams {
 
 // ---------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
+
+// One parameter's update from its mean gradient `grad` (Algorithm 2: Assistant.update).  SGD: param - lr * grad.
+// Adam (the optimizer the paper trained the Assistant with, Sec. 6.1): biased moments in a.m / a.v, bias-corrected step.
+__device__ __forceinline__ float adam_update(const AdamArgs& a, float param, float grad, float lr, int64_t j) {
+    const float m = a.beta1 * a.m[j] + (1.0f - a.beta1) * grad;
+    const float v = a.beta2 * a.v[j] + (1.0f - a.beta2) * grad * grad;
+    a.m[j] = m;
+    a.v[j] = v;
+    return param - lr * (m * a.corr1) / (sqrtf(v * a.corr2) + a.eps);
+}
 
 __device__ __forceinline__ void latch(Control* ctl, int code) { atomicCAS(&ctl->status, 0, code); }
 

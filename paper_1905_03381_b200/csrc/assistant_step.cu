@@ -159,7 +159,7 @@ __global__ void __launch_bounds__(256) linear_apply_kernel(StepParams p, int par
         float t = 0.0f;
 #pragma unroll
         for (int k = 0; k < 8; ++k) t += share[k][lane];
-        p.w[j] = p.w[j] - scale * t;
+        p.w[j] = p.adam.on ? adam_update(p.adam, p.w[j], t / (float)m, p.lr, j) : p.w[j] - scale * t;
     }
     if (blockIdx.x == 0 && grp == 1) {
         // bias: the per-CTA residual sums sit behind the column partials
@@ -167,7 +167,7 @@ __global__ void __launch_bounds__(256) linear_apply_kernel(StepParams p, int par
         for (int q = lane; q < parts; q += 32) t += p.partials[(int64_t)parts * p.d_pad + q];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
-        if (lane == 0) p.b[0] = p.b[0] - scale * t;
+        if (lane == 0) p.b[0] = p.adam.on ? adam_update(p.adam, p.b[0], t / (float)m, p.lr, p.f.d) : p.b[0] - scale * t;
     }
 }
 
@@ -211,7 +211,11 @@ template <int LPR>
 __global__ void __launch_bounds__(256) csr_scatter_kernel(StepParams p) {
     const int64_t m = batch_size(p);
     if (m <= 0) return;
-    const float scale = -p.lr / (float)m;
+    // SGD adds -lr/M r_i val straight onto the weights; Adam needs the mean gradient itself, collected in the
+    // (cleared) partial buffer and applied by adam_dense_kernel.
+    const float scale = p.adam.on ? 1.0f / (float)m : -p.lr / (float)m;
+    float* w_dst = p.adam.on ? p.partials : p.w;
+    float* b_dst = p.adam.on ? p.partials + p.csr.d : p.b;
     const int gl = threadIdx.x % LPR;
     const int64_t groups = (int64_t)gridDim.x * (blockDim.x / LPR);
     const int64_t g0 = (int64_t)blockIdx.x * (blockDim.x / LPR) + threadIdx.x / LPR;
@@ -227,12 +231,24 @@ __global__ void __launch_bounds__(256) csr_scatter_kernel(StepParams p) {
         const int e0 = __ldg(p.csr.indptr + r), e1 = __ldg(p.csr.indptr + r + 1);
         for (int e = e0 + gl; e < e1; e += LPR) {
             const int c = __ldg(p.csr.col + e);
-            if ((unsigned long long)(unsigned int)c < (unsigned long long)p.csr.d) atomicAdd(p.w + c, step * __ldg(p.csr.val + e));
+            if ((unsigned long long)(unsigned int)c < (unsigned long long)p.csr.d) atomicAdd(w_dst + c, step * __ldg(p.csr.val + e));
         }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) bias_acc += __shfl_xor_sync(0xFFFFFFFFu, bias_acc, o);
-    if ((threadIdx.x & 31) == 0 && bias_acc != 0.0f) atomicAdd(p.b, bias_acc);
+    if ((threadIdx.x & 31) == 0 && bias_acc != 0.0f) atomicAdd(b_dst, bias_acc);
+}
+
+// Adam over every weight of the bag-of-words Assistant from the mean gradient in the partial buffer (a weight whose
+// gradient is zero still moves while its first moment decays).
+__global__ void __launch_bounds__(256) adam_dense_kernel(StepParams p) {
+    const int64_t m = batch_size(p);
+    if (m <= 0) return;
+    const int64_t d = p.csr.d;
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j <= d; j += (int64_t)gridDim.x * blockDim.x) {
+        float* param = j < d ? p.w + j : p.b;
+        *param = adam_update(p.adam, *param, p.partials[j], p.lr, j);
+    }
 }
 
 template <typename T, bool VEC>
@@ -277,6 +293,7 @@ aa_status launch_assistant_step_dense(aa_ctx_impl* c, const DenseFeat& f, const 
     p.w = w;
     p.b = b;
     p.partials = c->partials;
+    p.adam = c->adam;
     p.ctl = c->ctl;
     p.d_pad = (f.d + ve - 1) / ve * ve;
     if (vec) {
@@ -336,7 +353,13 @@ aa_status launch_assistant_step_csr(aa_ctx_impl* c, const CsrFeat& f, const int3
     p.w = w;
     p.b = b;
     p.residual = c->row_scratch;
+    p.partials = c->partials;
+    p.adam = c->adam;
     p.ctl = c->ctl;
+    if (p.adam.on) {
+        if (f.d + 1 > c->partial_floats) return AA_ERR_WORKSPACE;
+        if (cudaMemsetAsync(c->partials, 0, sizeof(float) * (size_t)(f.d + 1), c->stream) != cudaSuccess) return AA_ERR_CUDA;
+    }
     int lpr = 4;
     while (lpr < 32 && lpr * 4 <= f.mean_nnz) lpr <<= 1;
     const int64_t rows_per_cta = 256 / lpr;
@@ -356,6 +379,12 @@ aa_status launch_assistant_step_csr(aa_ctx_impl* c, const CsrFeat& f, const int3
     ++c->launches;
     if (cudaLaunchKernel(k2, dim3(grid), dim3(256), args, 0, c->stream) != cudaSuccess) return AA_ERR_CUDA;
     ++c->launches;
+    if (p.adam.on) {
+        const int64_t want = (f.d + 1 + 255) / 256;
+        const int agrid = (int)(want < c->sm_count * 8 ? want : c->sm_count * 8);
+        if (cudaLaunchKernel((const void*)adam_dense_kernel, dim3(agrid), dim3(256), args, 0, c->stream) != cudaSuccess) return AA_ERR_CUDA;
+        ++c->launches;
+    }
     return AA_OK;
 }
 

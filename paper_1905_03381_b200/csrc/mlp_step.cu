@@ -57,6 +57,7 @@ struct MlpStepParams {
     float* part;              // [splits][hidden][d_pad]
     int64_t d_pad;
     int n_chunks, splits;
+    AdamArgs adam;
     Control* ctl;
 };
 
@@ -415,7 +416,8 @@ __global__ void __launch_bounds__(256) mlp_apply_w1_kernel(MlpStepParams p) {
         const int64_t u = q / p.d, k = q - u * p.d;
         float g = 0.0f;
         for (int s = 0; s < p.splits; ++s) g += p.part[((int64_t)s * p.g.hidden + u) * p.d_pad + k];
-        const float w = p.W1[q] - scale * __ldg(p.w2 + u) * g;
+        const float w = p.adam.on ? adam_update(p.adam, p.W1[q], __ldg(p.w2 + u) * g / (float)m, p.lr, q)
+                                  : p.W1[q] - scale * __ldg(p.w2 + u) * g;
         p.W1[q] = w;
         p.W1_bf16[q] = __float2bfloat16_rn(w);
     }
@@ -434,13 +436,20 @@ __global__ void __launch_bounds__(kMaxHidden) mlp_apply_small_kernel(MlpStepPara
             g_b1 += in[kMaxHidden + u];
         }
         const float w2_old = p.w2[u];
-        p.b1[u] = p.b1[u] - scale * w2_old * g_b1;
-        p.w2[u] = w2_old - scale * g_w2;
+        const int64_t hd = (int64_t)p.g.hidden * p.d;      // moments: W1, then b1, w2, b2
+        if (p.adam.on) {
+            p.b1[u] = adam_update(p.adam, p.b1[u], w2_old * g_b1 / (float)m, p.lr, hd + u);
+            p.w2[u] = adam_update(p.adam, w2_old, g_w2 / (float)m, p.lr, hd + p.g.hidden + u);
+        } else {
+            p.b1[u] = p.b1[u] - scale * w2_old * g_b1;
+            p.w2[u] = w2_old - scale * g_w2;
+        }
     }
     if (u == 0) {
         float g_b2 = 0.0f;
         for (int c = 0; c < ctas; ++c) g_b2 += p.small[(int64_t)c * (2 * kMaxHidden + 1) + 2 * kMaxHidden];
-        p.b2[0] = p.b2[0] - scale * g_b2;
+        p.b2[0] = p.adam.on ? adam_update(p.adam, p.b2[0], g_b2 / (float)m, p.lr, (int64_t)p.g.hidden * p.d + 2 * p.g.hidden)
+                            : p.b2[0] - scale * g_b2;
     }
 }
 
@@ -488,6 +497,7 @@ aa_status launch_assistant_step_mlp(aa_ctx_impl* c, const MlpFeat& f, float* W1_
     p.part = c->mlp_part;
     p.d_pad = (f.d + kFeatChunk - 1) / kFeatChunk * kFeatChunk;
     p.n_chunks = (int)(p.d_pad / kFeatChunk);
+    p.adam = c->adam;
     p.ctl = c->ctl;
     int max_ctas = c->sm_count < kMaxMlpCtas ? c->sm_count : kMaxMlpCtas;
     if (p.n_chunks > max_ctas) return AA_ERR_UNSUPPORTED;

@@ -26,6 +26,7 @@ struct StepParams {
     float* residual;      // per batch row (CSR path)
     int64_t d_pad;
     int rows_per_block;
+    AdamArgs adam;
     Control* ctl;
 };
 

@@ -1,0 +1,154 @@
+"""aa_assistant_step_adam against the oracle: the oracle's gradients (pinned by finite differences) fed through the
+oracle's Adam rule (pinned against torch.optim.Adam), three steps in a row from the oracle's own state.
+
+Bars: parameters |p - p_ref| <= 1e-4 |p_ref| + 1e-4 rms(p_ref), as for the SGD step; moments the same with rms floors.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import aa_oracle as O
+from paper_1905_03381_b200 import binding as B
+from paper_1905_03381_b200 import build, workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+LR, B1, B2, EPS = 0.002, 0.9, 0.999, 1e-5
+
+
+@pytest.fixture(scope="module")
+def aa():
+    build.build()
+    ctx = B.AutoAssist(max_rows=1 << 16, max_d=1 << 15, max_hidden=256, device=DEV)
+    yield ctx
+    torch.cuda.synchronize()
+    assert ctx.aa_device_status() == B.AA_OK
+    ctx.close()
+
+
+def close(got, ref, what, rel=1e-4):
+    ref = np.asarray(ref, np.float64).reshape(-1)
+    got = np.asarray(got, np.float64).reshape(-1)
+    tol = rel * np.abs(ref) + rel * math.sqrt(float(np.mean(ref ** 2)) + 1e-300)
+    assert np.all(np.abs(got - ref) <= tol), (what, float(np.max(np.abs(got - ref) - tol)))
+
+
+@pytest.mark.parametrize("n,m,d,dtype,use_rows", [
+    (900, 900, 100, torch.float32, False), (5000, 3100, 3072, torch.bfloat16, True), (2000, 1500, 512, torch.float32, True),
+])
+def test_linear_dense_adam_steps(aa, n, m, d, dtype, use_rows):
+    rng = np.random.default_rng(n + d)
+    x = W.normal((n, d), 1.0, 30 + d, dtype, DEV)
+    w = W.normal((d,), 0.05, 31, torch.float32, DEV)
+    b = torch.full((1,), 0.2, device=DEV)
+    rows = np.sort(rng.permutation(n)[:m]).astype(np.int32) if use_rows else None
+    rows_t = None if rows is None else torch.from_numpy(rows).to(DEV)
+    feat = B.dense_features(x, row_idx=rows_t) if use_rows else B.dense_features(x[:m])
+    mom, var = torch.zeros(d + 1, device=DEV), torch.zeros(d + 1, device=DEV)
+    state = B.adam_state(mom, var, B1, B2, EPS)
+    p_ref = np.concatenate([w.cpu().numpy(), b.cpu().numpy()])
+    m_ref, v_ref = np.zeros(d + 1, np.float32), np.zeros(d + 1, np.float32)
+    xh = W.to_oracle(x)
+    for t in range(1, 4):
+        loss = (W.normal((m,), 1.0, 40 + t, torch.float32, DEV).abs() * 2).contiguous()
+        aa.aa_assistant_step_adam(feat, loss, B.linear_assistant(w, b), state, LR)
+        torch.cuda.synchronize()
+        f = loss.cpu().numpy()
+        z = O.labels(f, O.batch_mean(f))
+        s = O.score_dense(xh, p_ref[:d], p_ref[d], row_idx=rows, n_cand=m)
+        gw, gb = O.linear_grad_dense(xh, s, z, row_idx=rows)
+        p_ref, m_ref, v_ref = O.adam(p_ref, m_ref, v_ref, np.concatenate([gw, [gb]]), LR, B1, B2, EPS, t)
+        assert state.t == t
+    close(np.concatenate([w.cpu().numpy(), b.cpu().numpy()]), p_ref, "params")
+    close(mom.cpu().numpy(), m_ref, "m", rel=2e-4)
+    close(var.cpu().numpy(), v_ref, "v", rel=2e-4)
+    assert np.abs(w.cpu().numpy() - p_ref[:d]).max() < 1 and np.abs(p_ref[:d]).max() > 0
+
+
+def test_csr_adam_steps(aa):
+    n, d, m = 3000, 1 << 14, 1200
+    rng = np.random.default_rng(70)
+    lens = rng.integers(1, 60, n)
+    indptr = np.zeros(n + 1, np.int32); indptr[1:] = np.cumsum(lens)
+    col = rng.integers(0, d, int(indptr[-1])).astype(np.int32)
+    val = rng.integers(1, 4, int(indptr[-1])).astype(np.float32)
+    rows = np.sort(rng.permutation(n)[:m]).astype(np.int32)
+    w = W.normal((d,), 0.05, 72, torch.float32, DEV)
+    b = torch.full((1,), 0.1, device=DEV)
+    ti, tc, tv = (torch.from_numpy(a).to(DEV) for a in (indptr, col, val))
+    feat = B.csr_features(ti, tc, tv, d, row_idx=torch.from_numpy(rows).to(DEV))
+    mom, var = torch.zeros(d + 1, device=DEV), torch.zeros(d + 1, device=DEV)
+    state = B.adam_state(mom, var, B1, B2, EPS)
+    p_ref = np.concatenate([w.cpu().numpy(), b.cpu().numpy()])
+    m_ref, v_ref = np.zeros(d + 1, np.float32), np.zeros(d + 1, np.float32)
+    for t in range(1, 4):
+        loss = (W.normal((m,), 1.0, 80 + t, torch.float32, DEV).abs() * 3).contiguous()
+        aa.aa_assistant_step_adam(feat, loss, B.linear_assistant(w, b), state, LR)
+        torch.cuda.synchronize()
+        f = loss.cpu().numpy()
+        z = O.labels(f, O.batch_mean(f))
+        s = O.score_csr(indptr, col, val, p_ref[:d], p_ref[d], row_idx=rows, n_cand=m)
+        gw, gb = O.linear_grad_csr(indptr, col, val, d, s, z, row_idx=rows)
+        p_ref, m_ref, v_ref = O.adam(p_ref, m_ref, v_ref, np.concatenate([gw, [gb]]), LR, B1, B2, EPS, t)
+    close(np.concatenate([w.cpu().numpy(), b.cpu().numpy()]), p_ref, "params")
+    close(mom.cpu().numpy(), m_ref, "m", rel=2e-4)
+    close(var.cpu().numpy(), v_ref, "v", rel=2e-4)
+
+
+def test_mlp_adam_steps(aa):
+    n, m, d, hidden = 3000, 2200, 320, 64
+    rng = np.random.default_rng(5)
+    x = W.normal((n, d), 1.0, 90, torch.bfloat16, DEV)
+    W1, b1, w2, b2 = W.mlp_assistant(d, hidden, 91, DEV)
+    b1 = W.normal((hidden,), 0.2, 92, torch.float32, DEV)
+    W1b = W1.to(torch.bfloat16).contiguous()
+    rows = np.sort(rng.permutation(n)[:m]).astype(np.int32)
+    feat = B.dense_features(x, row_idx=torch.from_numpy(rows).to(DEV))
+    total = hidden * (d + 2) + 1
+    mom, var = torch.zeros(total, device=DEV), torch.zeros(total, device=DEV)
+    state = B.adam_state(mom, var, B1, B2, EPS)
+    P = {"W1": W1.cpu().numpy().copy(), "b1": b1.cpu().numpy().copy(), "w2": w2.cpu().numpy().copy(), "b2": float(b2.item())}
+    bits = W.to_oracle(W1b).copy()
+    m_ref, v_ref = np.zeros(total, np.float32), np.zeros(total, np.float32)
+    xh = W.to_oracle(x)
+    xs = x.float().double().cpu().numpy()[rows]
+    for t in range(1, 3):
+        # Each step starts from the oracle's state (parameters, bf16 copy and moments): a difference of one ulp in a master
+        # weight can flip its bf16 rounding, which would turn the next forward pass into a different problem.
+        slack = np.zeros((hidden, d))
+        W1.copy_(torch.from_numpy(P["W1"])); b1.copy_(torch.from_numpy(P["b1"])); w2.copy_(torch.from_numpy(P["w2"])); b2.fill_(P["b2"])
+        W1b.copy_(torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).reshape(hidden, d))
+        mom.copy_(torch.from_numpy(m_ref)); var.copy_(torch.from_numpy(v_ref))
+        loss = (W.normal((m,), 1.0, 95 + t, torch.float32, DEV).abs() * 2).contiguous()
+        aa.aa_assistant_step_adam(feat, loss, B.mlp_assistant(W1, W1b, b1, w2, b2), state, LR)
+        torch.cuda.synchronize()
+        f = loss.cpu().numpy()
+        ref = O.assistant_step_mlp(xh, f, P["W1"], bits, P["b1"], P["w2"], P["b2"], 0.0, row_idx=rows)   # lr 0: gradients only
+        gW1, gb1, gw2, gb2 = ref["grads"]
+        flat_p = np.concatenate([P["W1"].reshape(-1), P["b1"], P["w2"], [P["b2"]]]).astype(np.float32)
+        flat_g = np.concatenate([gW1.reshape(-1), gb1, gw2, [gb2]])
+        flat_p, m_ref, v_ref = O.adam(flat_p, m_ref, v_ref, flat_g, LR, B1, B2, EPS, t)
+        # What the W1 gradient may differ by: P = r [a > 0] is rounded to bf16 (2^-9 per term), and a pre-activation within
+        # 1e-4 of zero may switch its unit on or off.  Adam divides the step by sqrt(v_hat) + eps, so a gradient difference dg
+        # moves a weight by up to about lr * dg / (sqrt(v_hat) + eps) (never more than 2 lr): small gradients are amplified.
+        r = np.abs(O.sigmoid(ref["s"]) - ref["z"])
+        on, near = ref["a"] > 0, np.abs(ref["a"]) < 1e-4
+        w2a = np.abs(P["w2"].astype(np.float64))[:, None]
+        # (the bf16 roundings are independent: six standard deviations of their sum, each uniform within 2^-9 of its term)
+        dg = (6.0 * 2.0 ** -9 / math.sqrt(3.0) * np.sqrt(((r ** 2)[:, None] * on).T @ xs ** 2) + (r[:, None] * near).T @ np.abs(xs)) * w2a / m
+        v_hat = v_ref[:hidden * d].astype(np.float64).reshape(hidden, d) / (1.0 - B2 ** t)
+        slack = np.minimum(2.0 * LR, 2.0 * LR * dg / (np.sqrt(v_hat) + EPS))
+        P = {"W1": flat_p[:hidden * d].reshape(hidden, d).copy(), "b1": flat_p[hidden * d:hidden * d + hidden].copy(),
+             "w2": flat_p[hidden * d + hidden:hidden * d + 2 * hidden].copy(), "b2": float(flat_p[-1])}
+        bits = O.round_bf16(P["W1"])
+        got_W1 = W1.cpu().numpy()
+        tol = 1e-4 * np.abs(P["W1"]) + 1e-4 * math.sqrt(float(np.mean(P["W1"].astype(np.float64) ** 2))) + slack
+        assert np.all(np.abs(got_W1 - P["W1"]) <= tol), float(np.max(np.abs(got_W1 - P["W1"]) - tol))
+        assert float(np.mean(slack > 0.25 * LR)) < 0.05     # the amplified cases are rare: most weights are held to a small fraction of a step
+        close(b1.cpu().numpy(), P["b1"], "b1")
+        close(w2.cpu().numpy(), P["w2"], "w2")
+        close([b2.item()], [P["b2"]], "b2")
+        assert np.array_equal(W.to_oracle(W1b), O.round_bf16(got_W1))
+    assert np.abs(W1.cpu().numpy() - W.mlp_assistant(d, hidden, 91, "cpu")[0].numpy()).max() > 0.5 * LR   # Adam moves weights by about lr per step

@@ -540,3 +540,28 @@ def test_hard_shrinking_rule():
     assert abs(counts[2] / v.size - math.exp(-1.0)) < 0.01          # P(Exp(1) >= 1) = 1/e
     assert np.array_equal(O.compact(O.hard_shrink(v, 1.0)), np.nonzero(v >= np.float32(1.0))[0])
     assert O.sk_threshold(3.0, 1) == 3.0 and math.isclose(O.sk_threshold(3.0, 12), 0.25, rel_tol=1e-6)
+
+
+def test_adam_rule_matches_torch_and_closed_forms():
+    import torch
+
+    rng = np.random.default_rng(21)
+    p0 = rng.normal(size=37).astype(np.float32)
+    grads = [rng.normal(size=37) * 0.1 for _ in range(5)]
+    # library routine: torch.optim.Adam in float64 on the same gradients
+    tp = torch.tensor(p0.astype(np.float64), requires_grad=True)
+    opt = torch.optim.Adam([tp], lr=0.01, betas=(0.9, 0.999), eps=1e-8)
+    p, m, v = p0.copy(), np.zeros(37, np.float32), np.zeros(37, np.float32)
+    for t, g in enumerate(grads, 1):
+        tp.grad = torch.tensor(g)
+        opt.step()
+        p, m, v = O.adam(p, m, v, g, 0.01, 0.9, 0.999, 1e-8, t)
+        assert np.allclose(p, tp.detach().numpy(), rtol=2e-6, atol=2e-7)
+    # first step from zero moments: every coordinate moves by lr * g / (|g| + eps), i.e. lr * sign(g)
+    p1, m1, v1 = O.adam(np.zeros(4, np.float32), np.zeros(4, np.float32), np.zeros(4, np.float32),
+                        np.array([0.3, -2.0, 1e-3, -1e-3]), 0.05, 0.9, 0.999, 1e-12, 1)
+    assert np.allclose(p1, [-0.05, 0.05, -0.05, 0.05], rtol=1e-6)
+    assert np.allclose(m1, 0.1 * np.array([0.3, -2.0, 1e-3, -1e-3]), rtol=1e-6) and np.allclose(v1, 1e-3 * np.array([0.09, 4.0, 1e-6, 1e-6]), rtol=1e-4, atol=0)
+    # zero gradient with a live first moment still moves the parameter
+    p2, _, _ = O.adam(np.zeros(1, np.float32), np.array([0.5], np.float32), np.array([0.25], np.float32), np.zeros(1), 0.1, 0.9, 0.999, 1e-8, 3)
+    assert p2[0] < 0
