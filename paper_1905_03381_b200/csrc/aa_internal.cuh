@@ -15,7 +15,8 @@ struct Control {
     unsigned int done;     // CTAs of the running scan kernel that have finished
     unsigned int epoch;    // generation of the look-back flags; bumped by the last CTA of each scan
     int status;            // first device-side condition latched (aa_status), 0 = none
-    unsigned int pad[60];
+    unsigned int sums_in;  // CTAs of the running gradient kernel that have published their share of the loss sum
+    unsigned int pad[59];
 };
 static_assert(sizeof(Control) == 256, "control block is one 256-byte line group");
 

@@ -298,7 +298,10 @@ aa_status launch_assistant_step_dense(aa_ctx_impl* c, const DenseFeat& f, const 
     p.d_pad = (f.d + ve - 1) / ve * ve;
     if (vec) {
         int parts = 0;
-        aa_status st = launch_assistant_grad_dense_tma(c, p, &parts);
+        aa_status st = launch_assistant_grad_dense_mma(c, p, &parts);
+        if (st == AA_OK) return launch_linear_apply(c, p, parts);
+        if (st != AA_ERR_UNSUPPORTED) return st;
+        st = launch_assistant_grad_dense_tma(c, p, &parts);
         if (st == AA_OK) return launch_linear_apply(c, p, parts);
         if (st != AA_ERR_UNSUPPORTED) return st;
     }

@@ -26,6 +26,7 @@ struct StepParams {
     float* residual;      // per batch row (CSR path)
     int64_t d_pad;
     int rows_per_block;
+    double* loss_sums;    // per-CTA shares of the batch loss sum (matrix-instruction kernel)
     AdamArgs adam;
     Control* ctl;
 };
@@ -69,6 +70,8 @@ __device__ __forceinline__ long long batch_row(const StepParams& p, int64_t i) {
 
 // Adds the per-CTA partial sums in CTA order and applies  w <- w - lr * grad  (defined in assistant_step.cu).
 aa_status launch_linear_apply(aa_ctx_impl* c, const StepParams& p, int parts);
+// Matrix-instruction variant for aligned bf16 rows of 256..3072 features (a multiple of 16); AA_ERR_UNSUPPORTED otherwise.
+aa_status launch_assistant_grad_dense_mma(aa_ctx_impl* c, StepParams& p, int* parts_out);
 // Bulk-copy variant of the dense gradient kernel; AA_ERR_UNSUPPORTED when the shape does not fit its ring.
 aa_status launch_assistant_grad_dense_tma(aa_ctx_impl* c, StepParams& p, int* parts_out);
 
