@@ -23,6 +23,7 @@ constexpr int kMlpStages = 3;
 constexpr int kABytes = kSuperRows * 128;       // feature slice of one stage
 constexpr int kMaxHidden = 256;
 constexpr int kTmemCols = 512;
+constexpr int kGatherWarps = 4;                 // warps that issue the row gathers when a row list selects the rows
 
 struct MlpGeom {
     int hidden;
@@ -77,19 +78,25 @@ __device__ __forceinline__ void tile_pipe_init(TilePipe* tp, uint32_t acc_consum
 template <bool GATHER>
 __device__ __forceinline__ bool mlp_produce(TilePipe* tp, unsigned char* ring, const CUtensorMap* map_x, const CUtensorMap* map_w,
                                             const MlpGeom& g, unsigned int n_tiles, const int32_t* rows, long long n_list,
-                                            long long n_stored) {
+                                            long long n_stored, int part = 0) {
+    // Gathered rows are fetched by kGatherWarps warps (part = 0 .. kGatherWarps - 1), 64 rows each, one four-row
+    // gather per lane and stage: the gathers a single warp issues retire at only about one per 43 ns.  Part 0 is the
+    // producer proper (it also posts the expected bytes and loads W1); the others follow the same barriers.
     const int lane = threadIdx.x & 31;
+    const bool helper = part != 0;
     volatile int* abort_flag = &tp->abort_flag;
     int stage = 0, j = 0;
     uint32_t phase = 0;
     bool ok = true;
+    constexpr int kRowsPerPart = kSuperRows / kGatherWarps;
+    const bool gather_lane = lane < kRowsPerPart / 4;
     for (unsigned int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         const long long k0 = (long long)tile * kSuperRows;
-        int r[8];
-        if (GATHER) {
+        int r[4] = {0, 0, 0, 0};
+        if (GATHER && gather_lane) {
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                const long long k = k0 + lane * 8 + q;
+            for (int q = 0; q < 4; ++q) {
+                const long long k = k0 + part * kRowsPerPart + lane * 4 + q;
                 long long row = k < n_list ? (long long)rows[k] : 0;
                 if ((unsigned long long)row >= (unsigned long long)n_stored) row = 0;
                 r[q] = (int)row;
@@ -98,15 +105,15 @@ __device__ __forceinline__ bool mlp_produce(TilePipe* tp, unsigned char* ring, c
         for (int ks = 0; ks < g.k_slices; ++ks) {
             if (!mbar_wait(&tp->empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
             unsigned char* a_dst = ring + (size_t)stage * g.stage_bytes;
-            if (lane == 0) {
+            if (lane == 0 && !helper) {
                 mbar_arrive_expect_tx(&tp->full[stage], (uint32_t)kABytes + g.b_bytes);
                 tma_load_2d(a_dst + kABytes, map_w, ks * kSliceK, 0, &tp->full[stage]);
                 if (!GATHER) tma_load_2d(a_dst, map_x, ks * kSliceK, (int)k0, &tp->full[stage]);
             }
             if (GATHER) {
                 __syncwarp();
-                tma_gather4(a_dst + (lane * 8) * 128, map_x, ks * kSliceK, r[0], r[1], r[2], r[3], &tp->full[stage]);
-                tma_gather4(a_dst + (lane * 8 + 4) * 128, map_x, ks * kSliceK, r[4], r[5], r[6], r[7], &tp->full[stage]);
+                if (gather_lane)
+                    tma_gather4(a_dst + (part * kRowsPerPart + lane * 4) * 128, map_x, ks * kSliceK, r[0], r[1], r[2], r[3], &tp->full[stage]);
             }
             __syncwarp();
             ++j;

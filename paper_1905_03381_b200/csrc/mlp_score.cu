@@ -27,7 +27,7 @@ namespace aa {
 
 namespace {
 
-constexpr int kMlpThreads = 384;
+constexpr int kMlpThreads = 448;               // warps 12, 13 only help with row gathers
 constexpr int kEpiWarps = 8;
 
 struct ScoreControl {
@@ -86,6 +86,9 @@ mlp_score_shrink_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
     if (warp == 0) {
         if (!mlp_produce<GATHER>(tp, ring, &map_x, &map_w, mp.g, n_tiles, p.row_idx, p.n_cand, p.n_stored) && lane == 0)
             mlp_give_up(p, tp);
+    } else if (GATHER && (warp == 3 || warp >= 12)) {
+        if (!mlp_produce<GATHER>(tp, ring, &map_x, &map_w, mp.g, n_tiles, p.row_idx, p.n_cand, p.n_stored, warp == 3 ? 1 : warp - 10) && lane == 0)
+            mlp_give_up(p, tp);
     } else if (warp == 1) {
         if (!mlp_issue_mma(tp, ring, mp.g, n_tiles, tmem_base) && lane == 0) mlp_give_up(p, tp);
     } else if (warp == 2) {
@@ -112,7 +115,7 @@ mlp_score_shrink_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
             }
             warp_shrink_compact<kSuperRows / 32>(p, tile, epoch, kSuperRows / 32, sv);
         }
-    } else if (warp >= 4) {
+    } else if (warp >= 4 && warp < 12) {
         // ------------------------------------------------------------ epilogue
         const int quad = warp & 3;                  // TMEM lanes 32*quad .. +31 are this warp's
         const int acc = (warp - 4) >> 2;            // which of the two accumulators

@@ -27,7 +27,7 @@ namespace aa {
 
 namespace {
 
-constexpr int kStepMlpThreads = 384;
+constexpr int kStepMlpThreads = 448;          // warps 12, 13 only help with row gathers
 constexpr int kStepEpiWarps = 8;
 constexpr int kMaxMlpCtas = 192;              // bound on the grids below (workspace sizing)
 constexpr int kFeatChunk = 256;               // feature columns per CTA of the W1-gradient kernel
@@ -141,9 +141,12 @@ mlp_residual_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
 
     if (warp == 0) {
         if (!mlp_produce<GATHER>(tp, ring, &map_x, &map_w, p.g, n_tiles, p.row_idx, m, p.n_stored) && lane == 0) step_give_up(p, tp);
+    } else if (GATHER && (warp == 3 || warp >= 12)) {
+        if (!mlp_produce<GATHER>(tp, ring, &map_x, &map_w, p.g, n_tiles, p.row_idx, m, p.n_stored, warp == 3 ? 1 : warp - 10) && lane == 0)
+            step_give_up(p, tp);
     } else if (warp == 1) {
         if (!mlp_issue_mma(tp, ring, p.g, n_tiles, tmem_base) && lane == 0) step_give_up(p, tp);
-    } else if (warp >= 4) {
+    } else if (warp >= 4 && warp < 12) {
         // ------------------------------------------------------------ epilogue
         const int ew = warp - 4;
         const int quad = warp & 3, acc = ew >> 2;
@@ -290,20 +293,22 @@ mlp_w1_grad_kernel(const __grid_constant__ CUtensorMap map_pt, const __grid_cons
     int n_q = (int)((p.d - col0 + 63) / 64);           // 64-column feature chunks that exist
     if (n_q > 4) n_q = 4;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ producer
+    if (warp == 0 || (GATHER && (warp == 3 || warp >= 12))) {
+        // ------------------------------------------------------------ producer (warp 0) and, for gathered rows, three helpers:
+        // gather warp q fetches 64-column chunk q of every stage, sixteen four-row gathers (one per lane); warp 0 also posts
+        // the expected bytes and loads the P^T box.
+        const int part = warp == 0 ? 0 : (warp == 3 ? 1 : warp - 10);
         int stage = 0, j = 0;
         uint32_t phase = 0;
         bool ok = true;
-        const int grp = lane & 15, half = lane >> 4;
         for (int sl = 0; sl < n_slices; ++sl) {
             const int64_t i0 = (s_begin + sl) * kRowSlice;
             int r0 = 0, r1 = 0, r2 = 0, r3 = 0;
-            if (GATHER) {
+            if (GATHER && lane < 16) {
                 int rr[4];
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    const int64_t i = i0 + grp * 4 + q;
+                    const int64_t i = i0 + lane * 4 + q;
                     long long row = i < m ? (long long)p.row_idx[i] : 0;
                     if ((unsigned long long)row >= (unsigned long long)p.n_stored) row = 0;   // its P column is zero
                     rr[q] = (int)row;
@@ -313,7 +318,7 @@ mlp_w1_grad_kernel(const __grid_constant__ CUtensorMap map_pt, const __grid_cons
             if (!mbar_wait(&gp->empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
             unsigned char* pt_dst = ring + (size_t)stage * kStage;
             unsigned char* x_dst = pt_dst + kPtBytes;
-            if (lane == 0) {
+            if (lane == 0 && part == 0) {
                 mbar_arrive_expect_tx(&gp->full[stage], p.g.b_bytes + (uint32_t)n_q * kXChunkBytes);   // P^T box: hidden rows
                 tma_load_2d(pt_dst, &map_pt, (int)i0, 0, &gp->full[stage]);
                 if (!GATHER)
@@ -321,11 +326,8 @@ mlp_w1_grad_kernel(const __grid_constant__ CUtensorMap map_pt, const __grid_cons
             }
             if (GATHER) {
                 __syncwarp();
-#pragma unroll
-                for (int cq = 0; cq < 2; ++cq) {
-                    const int q = half * 2 + cq;
-                    if (q < n_q) tma_gather4(x_dst + q * kXChunkBytes + (grp * 4) * 128, &map_x, col0 + q * 64, r0, r1, r2, r3, &gp->full[stage]);
-                }
+                if (lane < 16 && part < n_q)
+                    tma_gather4(x_dst + part * kXChunkBytes + (lane * 4) * 128, &map_x, col0 + part * 64, r0, r1, r2, r3, &gp->full[stage]);
             }
             __syncwarp();
             ++j;
@@ -371,7 +373,7 @@ mlp_w1_grad_kernel(const __grid_constant__ CUtensorMap map_pt, const __grid_cons
         __syncwarp();
         const long long t0 = clock64();
         while (!mbar_try_wait(&gp->drain, 0) && clock64() - t0 < kWaitCycles) {}
-    } else if (warp >= 4) {
+    } else if (warp >= 4 && warp < 12) {
         // ------------------------------------------------------------ epilogue: this CTA's partial of G
         const int quad = warp & 3, acc = (warp - 4) >> 2;
         const int u = acc * 128 + quad * 32 + lane;                 // hidden unit
