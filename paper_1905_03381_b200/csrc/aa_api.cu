@@ -444,7 +444,7 @@ aa_status aa_device_status(aa_ctx* ctx, int32_t* latched) {
         // a scan that gave up may have left the ticket state half-used: re-arm everything
         const unsigned int zeros[4] = {0, 0, 0, 0};
         if (cudaMemcpyAsync(c->ctl, zeros, 2 * sizeof(unsigned int), cudaMemcpyHostToDevice, c->stream) != cudaSuccess ||
-            cudaMemsetAsync(&c->ctl->status, 0, sizeof(int) + sizeof(unsigned int), c->stream) != cudaSuccess ||   // status, sums_in
+            cudaMemsetAsync(&c->ctl->status, 0, sizeof(int) + 2 * sizeof(unsigned int), c->stream) != cudaSuccess ||   // status, sums_in, applied
             cudaStreamSynchronize(c->stream) != cudaSuccess)
             return AA_ERR_CUDA;
     }

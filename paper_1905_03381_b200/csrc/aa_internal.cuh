@@ -16,7 +16,8 @@ struct Control {
     unsigned int epoch;    // generation of the look-back flags; bumped by the last CTA of each scan
     int status;            // first device-side condition latched (aa_status), 0 = none
     unsigned int sums_in;  // CTAs of the running gradient kernel that have published their share of the loss sum
-    unsigned int pad[59];
+    unsigned int applied;  // CTAs of the running gradient kernel that have seen every CTA's partial sums
+    unsigned int pad[58];
 };
 static_assert(sizeof(Control) == 256, "control block is one 256-byte line group");
 

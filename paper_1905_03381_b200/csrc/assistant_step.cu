@@ -299,7 +299,7 @@ aa_status launch_assistant_step_dense(aa_ctx_impl* c, const DenseFeat& f, const 
     if (vec) {
         int parts = 0;
         aa_status st = launch_assistant_grad_dense_mma(c, p, &parts);
-        if (st == AA_OK) return launch_linear_apply(c, p, parts);
+        if (st == AA_OK) return parts > 0 ? launch_linear_apply(c, p, parts) : AA_OK;
         if (st != AA_ERR_UNSUPPORTED) return st;
         st = launch_assistant_grad_dense_tma(c, p, &parts);
         if (st == AA_OK) return launch_linear_apply(c, p, parts);

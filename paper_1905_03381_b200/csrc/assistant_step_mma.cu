@@ -21,7 +21,9 @@
 //                    meet in shared memory (mbarrier, bounded wait), every warp forms the 16
 //                    residuals r = sigmoid(s) - z, then adds r * x for its own 256 columns into
 //                    accumulator fragments that live in registers for the whole kernel.
-// CTAs write column sums to the partial buffer; linear_apply_kernel adds them and takes the step.
+// CTAs write column sums to the partial buffer; once all of them have (a cooperative launch keeps the
+// grid co-resident, the wait is bounded all the same) each CTA adds up a slice of the columns and
+// takes the SGD or Adam step for it, so the step is one launch.
 #include <cuda_bf16.h>
 
 #include "async_copy.cuh"
@@ -188,7 +190,7 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_mma_kernel(StepParam
         // weights as three bf16 planes, and the batch-mean threshold (fixed order: thread stride, warp tree, warp index)
         for (int jf = ct; jf < g.d; jf += kMWarps * 32) {
             __nv_bfloat16 hi, mid, lo;
-            split3(__ldg(p.f.w + jf), hi, mid, lo);
+            split3(__ldcg(p.f.w + jf), hi, mid, lo);       // w is rewritten at the end of this kernel: no read-only path
             w_split[jf] = hi;
             w_split[g.d + jf] = mid;
             w_split[2 * g.d + jf] = lo;
@@ -358,15 +360,65 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_mma_kernel(StepParam
         }
     }
     __syncthreads();
+    // ---------------------------------------------------------------- update (Algorithm 2: Assistant.update)
+    // Every CTA publishes its sums, waits (bounded) until all CTAs of this cooperative launch have done so, then adds
+    // the partial sums of its own slice of the columns in a fixed order and takes the step for that slice.
     if (tid == 0) {
         p.partials[(int64_t)gridDim.x * p.d_pad + blockIdx.x] = cb->bias_sum;
-        // last CTA out re-arms the ticket counter for the next kernel on this context
         __threadfence();
-        const unsigned int prev = atomicAdd(&p.ctl->done, 1u);
-        if (prev == gridDim.x - 1) {
-            p.ctl->ticket = 0;
-            p.ctl->done = 0;
-            p.ctl->sums_in = 0;
+        atomicAdd(&p.ctl->done, 1u);
+        unsigned int polls = 0;
+        while (*(volatile unsigned int*)&p.ctl->done < gridDim.x && !*abort_flag) {
+            if (++polls > kSpinLimit) break;
+            __nanosleep(64);
+        }
+        if (*(volatile unsigned int*)&p.ctl->done < gridDim.x || *abort_flag) {
+            mma_give_up(p, cb);
+        } else {
+            __threadfence();
+            // the last CTA past the wait re-arms the counters for the next kernel on this context
+            const unsigned int prev = atomicAdd(&p.ctl->applied, 1u);
+            if (prev == gridDim.x - 1) {
+                p.ctl->ticket = 0;
+                p.ctl->done = 0;
+                p.ctl->sums_in = 0;
+                p.ctl->applied = 0;
+            }
+        }
+    }
+    __syncthreads();
+    if (*abort_flag || m <= 0) return;
+    {
+        float* share = reinterpret_cast<float*>(x_ring);            // [warps][32]; every copy into the ring has landed
+        constexpr int kAllWarps = kMThreads / 32;
+        const int cols_per_cta = (g.d + (int)gridDim.x - 1) / (int)gridDim.x;
+        const int c0 = (int)blockIdx.x * cols_per_cta;
+        const int c1 = c0 + cols_per_cta < g.d ? c0 + cols_per_cta : g.d;
+        const float scale = p.lr / (float)m;
+        for (int cb0 = c0; cb0 < c1; cb0 += 32) {
+            const int jcol = cb0 + lane;
+            float gsum = 0.0f;
+            if (jcol < c1) {
+#pragma unroll 4
+                for (unsigned int q = warp; q < gridDim.x; q += kAllWarps) gsum += __ldcg(p.partials + (int64_t)q * p.d_pad + jcol);
+            }
+            share[warp * 32 + lane] = gsum;
+            __syncthreads();
+            if (warp == 0 && jcol < c1) {
+                float t = 0.0f;
+#pragma unroll
+                for (int k = 0; k < kAllWarps; ++k) t += share[k * 32 + lane];
+                const float w_old = __ldcg(p.w + jcol);
+                p.w[jcol] = p.adam.on ? adam_update(p.adam, w_old, t / (float)m, p.lr, jcol) : w_old - scale * t;
+            }
+            __syncthreads();
+        }
+        if (blockIdx.x == 0 && warp == 1) {
+            float t = 0.0f;
+            for (unsigned int q = lane; q < gridDim.x; q += 32) t += __ldcg(p.partials + (int64_t)gridDim.x * p.d_pad + q);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
+            if (lane == 0) p.b[0] = p.adam.on ? adam_update(p.adam, p.b[0], t / (float)m, p.lr, p.f.d) : p.b[0] - scale * t;
         }
     }
 }
@@ -396,9 +448,10 @@ aa_status launch_assistant_grad_dense_mma(aa_ctx_impl* c, StepParams& p, int* pa
     const void* kernel = (const void*)linear_grad_mma_kernel;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return AA_ERR_CUDA;
     void* args[] = {&p, &g};
-    if (cudaLaunchKernel(kernel, dim3(grid), dim3(kMThreads), args, smem, c->stream) != cudaSuccess) return AA_ERR_CUDA;
+    // cooperative: the CTAs wait for one another before the update, so all of them must be resident at once
+    if (cudaLaunchCooperativeKernel(kernel, dim3(grid), dim3(kMThreads), args, smem, c->stream) != cudaSuccess) return AA_ERR_CUDA;
     ++c->launches;
-    *parts_out = grid;
+    *parts_out = 0;   // the update was taken inside the kernel
     return AA_OK;
 }
 

@@ -71,6 +71,7 @@ __device__ __forceinline__ long long batch_row(const StepParams& p, int64_t i) {
 // Adds the per-CTA partial sums in CTA order and applies  w <- w - lr * grad  (defined in assistant_step.cu).
 aa_status launch_linear_apply(aa_ctx_impl* c, const StepParams& p, int parts);
 // Matrix-instruction variant for aligned bf16 rows of 256..3072 features (a multiple of 16); AA_ERR_UNSUPPORTED otherwise.
+// *parts_out = 0 when the kernel has taken the update itself (no apply launch needed).
 aa_status launch_assistant_grad_dense_mma(aa_ctx_impl* c, StepParams& p, int* parts_out);
 // Bulk-copy variant of the dense gradient kernel; AA_ERR_UNSUPPORTED when the shape does not fit its ring.
 aa_status launch_assistant_grad_dense_tma(aa_ctx_impl* c, StepParams& p, int* parts_out);
