@@ -43,6 +43,9 @@ def parse_args():
     ap.add_argument("--pool-rows", type=int, default=None, help="override the pool size (testing only)")
     ap.add_argument("--workload", default="image", choices=["image", "mlp"],
                     help="image = the benchmark workload; mlp = the two-layer (tensor-core) Assistant shape")
+    ap.add_argument("--pipeline-steps", type=int, default=300,
+                    help="steps of the two-stream Assistant/Boss schedule timed after the main region (0 = skip)")
+    ap.add_argument("--pipeline-depth", type=int, default=2, help="Boss queue depth k of that schedule")
     ap.add_argument("--loss-reps", type=int, default=20,
                     help="timed calls of the per-sentence loss on the translation shape (0 = skip)")
     return ap.parse_args()
@@ -306,6 +309,46 @@ def run_b200(args, cfg):
 
     agg = sharding.aggregate(dist if world > 1 else None, dev, elapsed_ms, cfg.n * K)
 
+    # ---- the same three stages as the two-stream schedule with a Boss queue of depth k (screening runs ahead of the
+    # losses and updates it no longer waits for); reported beside the sequential figure, which stays the metric
+    pipeline = None
+    if args.pipeline_steps > 0 and world == 1:
+        from paper_1905_03381_b200.pipeline import StreamPipeline
+
+        pipe = StreamPipeline(args.pipeline_depth, max_rows=cfg.n, max_d=cfg.d, capacity=cfg.n, device=dev)
+        gathered = {}
+
+        def features(j, row_idx):
+            kk = j % npool
+            if row_idx is None:
+                return feats[kk]
+            key = (kk, row_idx.data_ptr())
+            if key not in gathered:
+                gathered[key] = B.dense_features(pools[kk], row_idx=row_idx, id_base=plan.id_bases[kk])
+            return gathered[key]
+
+        def boss(t, ctx, idx, count_dev, out_loss):
+            ctx.aa_instance_loss(lg[t % npool], labels[t % npool], out_loss, count_dev=count_dev)
+
+        P = args.pipeline_steps
+        pipe.run(max(args.warmup, 3), features, boss, asst, cfg.gamma, cfg.philox_seed, cfg.lr, first_step=5000)
+        torch.cuda.synchronize()
+        n0 = pipe.launch_count()
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        p0.record()
+        pipe.run(P, features, boss, asst, cfg.gamma, cfg.philox_seed, cfg.lr, first_step=6000)
+        p1.record()
+        torch.cuda.synchronize()
+        pst = pipe.device_status()
+        assert pst == B.AA_OK, B.status_string(pst)
+        pms = p0.elapsed_time(p1) / P
+        pipeline = {"schedule": "Assistant stream: screen pool t+k, update on batch t; Boss stream: losses of batch t; "
+                                "batch j screened with the parameters after max(0, j-k) updates",
+                    "depth": args.pipeline_depth, "steps": P, "ms_per_step": pms, "value": cfg.n / (pms * 1e-3), "unit": UNIT,
+                    "gpu_launches": int(pipe.launch_count() - n0)}
+        pipe.close()
+        del pipe
+
     # ---- second half of the metric: per-instance-loss rows/s on the translation shape
     # (25,000 token rows x 32,000-word bf16 logits = 1.6 GB per call, larger than L2; per-sentence sums)
     loss_rows = None
@@ -406,7 +449,7 @@ def run_b200(args, cfg):
         "metric": METRIC, "value": agg["units"] / (agg["ms"] * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": max(args.warmup, 3), "ms_per_step": agg["ms"] / K, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(cfg, args),
-        "roofline": roofline, "stages": stages, "instance_loss_rows": loss_rows, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
+        "roofline": roofline, "stages": stages, "instance_loss_rows": loss_rows, "pipeline": pipeline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
         "accepted_mean": accepted, "accepted_min": int(timed.min()), "accepted_max": int(timed.max()), "clocks": sampler.summary(),
     }
     print(json.dumps(line), flush=True)

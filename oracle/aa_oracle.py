@@ -375,3 +375,43 @@ def adam(param, m, v, grad, lr: float, beta1: float, beta2: float, eps: float, t
         v_hat = v_new[j] / (1.0 - b2 ** t)
         p_new[j] = p64[j] - lr * m_hat / (np.sqrt(v_hat) + float(np.float32(eps)))
     return p_new.astype(np.float32), m_new.astype(np.float32), v_new.astype(np.float32)
+
+
+def pipeline_linear_dense(pool_of, logits_of, w, b, gamma: float, seed: int, lr: float, depth: int, n_steps: int, T=None):
+    """The Assistant / Boss schedule of Sec. 5.3 (Algorithms 2 and 3) with a Boss queue of `depth` batches, written
+    as the one sequence of events it becomes when both workers take turns in a fixed order:
+
+      Assistant: while the Boss queue is short (fewer than `depth` batches ahead of the Boss, and always the batch the
+                 Boss needs next), screen the next pool with the CURRENT parameters and enqueue its batch;
+      Boss:      pop batch t, evaluate its per-instance losses, push (batch, losses) to the Assistant queue;
+      Assistant: pop that item, take one update.
+
+    So batch j is screened with the parameters after max(0, j - depth) updates; depth = 0 is the sequential path.
+    pool_of(j) -> feature matrix of pool j (bf16 bits or fp32); logits_of(j) -> (logits, labels) whose row i belongs
+    to the i-th instance of batch j.  Batch j is screened with Philox step j.
+    Returns a list of per-step dicts {B, f, w, b} (w, b = parameters after that step's update) and the list `lag`
+    with lag[j] = number of updates the parameters had seen when batch j was screened.
+    """
+    w_cur = np.array(w, np.float32, copy=True)
+    b_cur = np.float32(b)
+    queue = {}
+    lag = []
+    updates = 0
+    next_screen = 0
+    out = []
+    for t in range(n_steps):
+        # Assistant: sampling has priority over updating while the Boss queue is short
+        while next_screen < n_steps and next_screen <= t + depth:
+            r = screen_linear_dense(pool_of(next_screen), w_cur, b_cur, gamma, seed, next_screen)
+            queue[next_screen] = r["B"]
+            lag.append(updates)
+            next_screen += 1
+        # Boss: losses of batch t
+        Bt = queue.pop(t)
+        lg, lab = logits_of(t)
+        f = instance_loss(lg[: len(Bt)], np.asarray(lab)[: len(Bt)])
+        # Assistant: one update on (batch t, losses)
+        w_cur, b_cur, _ = assistant_step_linear_dense(pool_of(t), f, w_cur, b_cur, lr, T=T, row_idx=np.asarray(Bt, np.int32))
+        updates += 1
+        out.append({"B": Bt, "f": f, "w": w_cur.copy(), "b": np.float32(b_cur)})
+    return out, lag

@@ -1,0 +1,122 @@
+"""The two-stream Assistant / Boss schedule (Sec. 5.3, Algorithms 2-3) against the CPU oracle.
+
+Bars:
+  * schedule: batch j equals the oracle's screening of pool j with the parameters the GPU held after
+    max(0, j - depth) updates, bit for bit outside the tie band |p - c| < 1e-5;
+  * losses: abs 1e-4 per row; parameters after update t (from the GPU's own state before it):
+    |w - w_ref| <= 1e-4 |w_ref| + 1e-4 rms(w_ref);
+  * free-running oracle schedule from the same start: identical batches up to the first step that holds a
+    candidate inside the tie band.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import aa_oracle as O
+from paper_1905_03381_b200 import binding as B
+from paper_1905_03381_b200 import build, workloads as W
+from paper_1905_03381_b200.pipeline import StreamPipeline
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+N, D, CLASSES, STEPS = 4096 + 77, 256, 100, 6
+MIX, SEED, LR = 0.15, 123, 2.0
+
+
+@pytest.fixture(scope="module")
+def data():
+    build.build()
+    pools = [W.normal((N, D), 1.0, 500 + j, torch.bfloat16, DEV) for j in range(STEPS)]
+    logits = [W.normal((N, CLASSES), 3.0, 600 + j, torch.float32, DEV) for j in range(STEPS)]
+    labels = [W.randint(0, CLASSES, (N,), 700 + j, DEV).to(torch.int32) for j in range(STEPS)]
+    w0 = W.normal((D,), 0.05, 9, torch.float32, DEV)
+    return pools, logits, labels, w0
+
+
+def run_gpu(data, depth):
+    pools, logits, labels, w0 = data
+    w = w0.clone()
+    b = torch.full((1,), 0.1, dtype=torch.float32, device=DEV)
+    assistant = B.linear_assistant(w, b)
+    pipe = StreamPipeline(depth, max_rows=N, max_d=D, capacity=N, device=DEV, slots=STEPS)
+    w_hist = torch.zeros((STEPS, D), dtype=torch.float32, device=DEV)
+    b_hist = torch.zeros((STEPS, 1), dtype=torch.float32, device=DEV)
+
+    def features(j, row_idx):
+        return B.dense_features(pools[j], row_idx=row_idx)
+
+    def boss(t, ctx, idx, count_dev, out_loss):
+        ctx.aa_instance_loss(B.logits_desc(logits[t]), labels[t], out_loss, count_dev=count_dev)
+
+    def after_update(t):
+        w_hist[t].copy_(w)
+        b_hist[t].copy_(b)
+
+    pipe.run(STEPS, features, boss, assistant, MIX, SEED, LR, after_update=after_update)
+    torch.cuda.synchronize()
+    assert pipe.device_status() == B.AA_OK
+    assert pipe.launch_count() >= 3 * STEPS
+    out = {"idx": pipe.idx.cpu().numpy(), "count": pipe.count.cpu().numpy()[:, 0], "loss": pipe.loss.cpu().numpy(),
+           "w": w_hist.cpu().numpy(), "b": b_hist.cpu().numpy()[:, 0]}
+    pipe.close()
+    return out
+
+
+@pytest.mark.parametrize("depth", [0, 1, 3])
+def test_schedule_matches_oracle(data, depth):
+    pools, logits, labels, w0 = data
+    g = run_gpu(data, depth)
+    pools_h = [W.to_oracle(p) for p in pools]
+    logits_h = [l.cpu().numpy() for l in logits]
+    labels_h = [l.cpu().numpy() for l in labels]
+    w0_h = w0.cpu().numpy()
+    snaps = [(w0_h, np.float32(0.1))] + [(g["w"][t], np.float32(g["b"][t])) for t in range(STEPS)]
+    ids = np.arange(N)
+    for j in range(STEPS):
+        wj, bj = snaps[max(0, j - depth)]
+        ref = O.screen_linear_dense(pools_h[j], wj, bj, MIX, SEED, j)
+        c = O.uniform(SEED, j, ids)
+        m = int(g["count"][j])
+        got = np.zeros(N, np.uint8)
+        got[g["idx"][j][:m]] = 1
+        assert np.all(np.diff(g["idx"][j][:m]) > 0)
+        differ = got != ref["keep"]
+        assert np.all(np.abs(ref["p"] - c)[differ] < 1e-5), f"batch {j}: decisions differ outside the tie band"
+        # a wrong lag would show: the neighbouring snapshots give other batches once the parameters have moved
+        if depth and j > depth:
+            other = O.screen_linear_dense(pools_h[j], *snaps[j], MIX, SEED, j)
+            assert not np.array_equal(other["keep"], ref["keep"])
+    for t in range(STEPS):
+        m = int(g["count"][t])
+        Bt = g["idx"][t][:m].astype(np.int32)
+        f_ref = O.row_loss(logits_h[t][:m], labels_h[t][:m])
+        assert np.all(np.abs(g["loss"][t][:m] - f_ref) <= 1e-4)
+        w_ref, b_ref, _ = O.assistant_step_linear_dense(pools_h[t], g["loss"][t][:m], snaps[t][0], snaps[t][1], LR, row_idx=Bt)
+        rms = float(np.sqrt(np.mean(w_ref.astype(np.float64) ** 2)))
+        assert np.all(np.abs(g["w"][t] - w_ref) <= 1e-4 * np.abs(w_ref) + 1e-4 * rms)
+        assert abs(g["b"][t] - b_ref) <= 1e-4 * abs(b_ref) + 1e-4 * rms
+    # free-running oracle from the same start
+    free, lag = O.pipeline_linear_dense(lambda j: pools_h[j], lambda j: (logits_h[j], labels_h[j]), w0_h, 0.1, MIX, SEED, LR,
+                                        depth, STEPS)
+    assert lag == [max(0, j - depth) for j in range(STEPS)]
+    for j in range(STEPS):
+        wj, bj = ((w0_h, np.float32(0.1)) if lag[j] == 0 else (free[lag[j] - 1]["w"], free[lag[j] - 1]["b"]))
+        p = O.screen_linear_dense(pools_h[j], wj, bj, MIX, SEED, j)["p"]
+        if np.any(np.abs(p - O.uniform(SEED, j, ids)) < 1e-5):
+            break
+        assert np.array_equal(free[j]["B"], g["idx"][j][: int(g["count"][j])])
+
+
+def test_depth_changes_batches_and_reruns_agree(data):
+    a = run_gpu(data, 0)
+    b1 = run_gpu(data, 2)
+    b2 = run_gpu(data, 2)
+    # stale screening is visible at this learning rate, and the overlap of the two streams changes nothing
+    assert any(a["count"][j] != b1["count"][j] or not np.array_equal(a["idx"][j], b1["idx"][j]) for j in range(3, STEPS))
+    # (the gradient's summation order is not fixed between runs, so a candidate on the very edge of its decision may flip)
+    for j in range(STEPS):
+        s1 = set(b1["idx"][j][: int(b1["count"][j])].tolist())
+        s2 = set(b2["idx"][j][: int(b2["count"][j])].tolist())
+        assert len(s1 ^ s2) <= 2
+    # batches 0..2 were screened before the first update in both runs of depth 2, batch 0 in every run
+    assert np.array_equal(a["idx"][0][: int(a["count"][0])], b1["idx"][0][: int(b1["count"][0])])

@@ -565,3 +565,50 @@ def test_adam_rule_matches_torch_and_closed_forms():
     # zero gradient with a live first moment still moves the parameter
     p2, _, _ = O.adam(np.zeros(1, np.float32), np.array([0.5], np.float32), np.array([0.25], np.float32), np.zeros(1), 0.1, 0.9, 0.999, 1e-8, 3)
     assert p2[0] < 0
+
+
+def _pipeline_inputs(n_steps, n=300, d=12, classes=5, seed=31):
+    rng = np.random.default_rng(seed)
+    pools = [rng.normal(size=(n, d)).astype(np.float32) for _ in range(n_steps)]
+    logits = [rng.normal(size=(n, classes)).astype(np.float32) * 2 for _ in range(n_steps)]
+    labels = [rng.integers(0, classes, n).astype(np.int32) for _ in range(n_steps)]
+    w0 = (rng.normal(size=d) * 0.3).astype(np.float32)
+    return pools, logits, labels, w0
+
+
+def test_pipeline_schedule_lag_and_special_cases():
+    """Sec. 5.3 / Algorithms 2-3 as one event sequence: batch j is screened with the parameters after
+    max(0, j - depth) updates; depth 0 is the plain chain screen -> loss -> update; a zero learning rate makes the
+    depth irrelevant; batches screened before the first update do not depend on the learning rate."""
+    steps = 7
+    pools, logits, labels, w0 = _pipeline_inputs(steps)
+    pool_of = lambda j: pools[j]
+    logits_of = lambda j: (logits[j], labels[j])
+    runs = {}
+    for depth in (0, 1, 3, 10):
+        out, lag = O.pipeline_linear_dense(pool_of, logits_of, w0, 0.05, 0.2, 77, 0.5, depth, steps)
+        assert lag == [max(0, j - depth) for j in range(steps)]
+        runs[depth] = out
+        # batch j against a screening with the snapshot the lag names (snapshots come from the run itself)
+        snaps = [(w0, np.float32(0.05))] + [(o["w"], o["b"]) for o in out]
+        for j in range(steps):
+            wj, bj = snaps[lag[j]]
+            assert np.array_equal(out[j]["B"], O.screen_linear_dense(pools[j], wj, bj, 0.2, 77, j)["B"])
+    # depth 0 == the chain written out by hand
+    w, b = w0.copy(), np.float32(0.05)
+    for t in range(steps):
+        Bt = O.screen_linear_dense(pools[t], w, b, 0.2, 77, t)["B"]
+        f = O.row_loss(logits[t][: len(Bt)], labels[t][: len(Bt)])
+        w, b, _ = O.assistant_step_linear_dense(pools[t], f, w, b, 0.5, row_idx=Bt.astype(np.int32))
+        assert np.array_equal(Bt, runs[0][t]["B"]) and np.array_equal(w, runs[0][t]["w"]) and b == runs[0][t]["b"]
+    # a learning rate that moves the parameters makes stale screening visible: some later batch differs between depths
+    assert any(not np.array_equal(runs[0][t]["B"], runs[3][t]["B"]) for t in range(1, steps))
+    # the first depth+1 batches are screened before any update: identical to depth 10 (all screened with the initial parameters)
+    for t in range(4):
+        assert np.array_equal(runs[3][t]["B"], runs[10][t]["B"])
+    # lr = 0: every depth gives the same batches, and the parameters never move
+    base, _ = O.pipeline_linear_dense(pool_of, logits_of, w0, 0.05, 0.2, 77, 0.0, 0, steps)
+    for depth in (1, 4):
+        other, _ = O.pipeline_linear_dense(pool_of, logits_of, w0, 0.05, 0.2, 77, 0.0, depth, steps)
+        for t in range(steps):
+            assert np.array_equal(base[t]["B"], other[t]["B"]) and np.array_equal(other[t]["w"], w0)
