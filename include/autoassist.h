@@ -248,6 +248,19 @@ aa_status aa_instance_loss(aa_ctx* ctx, const aa_logits* logits, const int32_t* 
                            float* out_loss);
 
 /*
+ * Step 4 on a batch list: the Boss losses of the batch instances when the logits (and labels) are
+ * stored for the whole pool (Sec. 5.3: the losses {f(x_i, y_i)} of the instances i in B).
+ *   out_loss[k] = l_r with r = row_idx[k], for k in [0, M), M = min(*count_dev, n_rows) when
+ *   count_dev is given, else n_rows; labels[r] is the label of stored row r.
+ * row_idx: device int32 list (e.g. out_idx of aa_score_shrink); an entry outside [0, logits->rows)
+ * gives 0 and latches AA_ERR_BAD_INDEX.  Label rules as in aa_instance_loss.  out_loss holds
+ * n_rows entries; entries at and beyond M are left untouched.
+ */
+aa_status aa_instance_loss_rows(aa_ctx* ctx, const aa_logits* logits, const int32_t* labels,
+                                const int32_t* row_idx, int64_t n_rows, const int32_t* count_dev,
+                                float* out_loss);
+
+/*
  * Step 5: labels and one SGD step of the Assistant on the batch (Algorithm 2: gradient, update).
  * Batch instance i is stored row feat->row_idx[i] (or row i), i in [0, M), M = min(*count_dev,
  * feat->n_rows) when count_dev is given, else feat->n_rows (or feat->n without row_idx).

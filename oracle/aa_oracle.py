@@ -415,3 +415,13 @@ def pipeline_linear_dense(pool_of, logits_of, w, b, gamma: float, seed: int, lr:
         updates += 1
         out.append({"B": Bt, "f": f, "w": w_cur.copy(), "b": np.float32(b_cur)})
     return out, lag
+
+
+def instance_loss_rows(logits, labels, row_idx) -> np.ndarray:
+    """Losses of the batch instances (Sec. 5.3: {f(x_i, y_i)} for i in B) out of logits / labels stored for the whole
+    pool: entry k is the row loss of stored row row_idx[k]."""
+    labels = _arr(labels, np.int32)
+    out = np.zeros(len(row_idx), dtype=np.float64)
+    for k, r in enumerate(np.asarray(row_idx, dtype=np.int64)):
+        out[k] = row_loss(logits[r: r + 1], labels[r: r + 1])[0]
+    return out

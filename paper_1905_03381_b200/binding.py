@@ -27,6 +27,7 @@ EXPORTS = (
     "aa_status_string", "aa_workspace_bytes", "aa_create", "aa_destroy", "aa_score_shrink",
     "aa_shrink_compact", "aa_instance_loss", "aa_assistant_step", "aa_step_host_staging_bytes", "aa_step_host",
     "aa_device_status", "aa_launch_count", "aa_shrink_compact_static", "aa_batch_cut", "aa_threshold_compact", "aa_sk_threshold", "aa_assistant_step_adam",
+    "aa_instance_loss_rows",
 )
 AA_STATIC_MAX_CANDIDATES = 1 << 22
 
@@ -109,6 +110,7 @@ def lib() -> ctypes.CDLL:
         L.aa_batch_cut.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_int64, c_int64,
                                    c_void_p, c_void_p, c_void_p, c_int64]
         L.aa_instance_loss.argtypes = [c_void_p, POINTER(aa_logits), c_void_p, c_void_p, c_int64, c_void_p, c_void_p]
+        L.aa_instance_loss_rows.argtypes = [c_void_p, POINTER(aa_logits), c_void_p, c_void_p, c_int64, c_void_p, c_void_p]
         L.aa_assistant_step.argtypes = [c_void_p, POINTER(aa_feat), c_void_p, c_void_p, POINTER(aa_assistant),
                                         c_float, c_int32, c_float]
         L.aa_step_host_staging_bytes.argtypes = [POINTER(aa_feat), POINTER(aa_logits), POINTER(c_size_t)]
@@ -303,6 +305,14 @@ class AutoAssist:
         self._ok(self._L.aa_instance_loss(self._ctx, byref(logits), labels.data_ptr(), _ptr(offsets),
                                           0 if n_seg is None else n_seg, _ptr(count_dev), out_loss.data_ptr()),
                  "aa_instance_loss")
+
+    def aa_instance_loss_rows(self, logits: aa_logits, labels: torch.Tensor, row_idx: torch.Tensor, out_loss: torch.Tensor,
+                              count_dev=None, n_rows=None):
+        """Losses of the batch instances row_idx[k] out of logits / labels stored for the whole pool."""
+        _check(row_idx, torch.int32, "row_idx")
+        self._ok(self._L.aa_instance_loss_rows(self._ctx, byref(logits), labels.data_ptr(), row_idx.data_ptr(),
+                                               row_idx.numel() if n_rows is None else n_rows, _ptr(count_dev),
+                                               out_loss.data_ptr()), "aa_instance_loss_rows")
 
     def aa_assistant_step(self, feat: aa_feat, loss: torch.Tensor, assistant: aa_assistant, lr: float,
                           threshold=None, count_dev=None):

@@ -291,6 +291,17 @@ aa_status aa_instance_loss(aa_ctx* ctx, const aa_logits* lg, const int32_t* labe
     return launch_instance_loss(c, *lg, labels, offsets, n_seg, count_dev, out_loss);
 }
 
+aa_status aa_instance_loss_rows(aa_ctx* ctx, const aa_logits* lg, const int32_t* labels, const int32_t* row_idx, int64_t n_rows,
+                                const int32_t* count_dev, float* out_loss) {
+    if (!ctx || !lg || lg->rows < 0 || lg->cols <= 0 || lg->row_stride < lg->cols || n_rows < 0) return AA_ERR_INVALID_ARG;
+    if (lg->dtype != AA_F32 && lg->dtype != AA_BF16) return AA_ERR_INVALID_ARG;
+    if (n_rows > 0 && (!lg->data || !labels || !row_idx || !out_loss)) return AA_ERR_INVALID_ARG;
+    if ((uintptr_t)lg->data % (lg->dtype == AA_BF16 ? 2 : 4)) return AA_ERR_INVALID_ARG;
+    if (lg->cols > 0x7FFFFFFFll) return AA_ERR_INVALID_ARG;
+    if (n_rows == 0) return AA_OK;
+    return launch_instance_loss(&ctx->impl, *lg, labels, nullptr, 0, count_dev, out_loss, row_idx, n_rows);
+}
+
 aa_status aa_assistant_step(aa_ctx* ctx, const aa_feat* feat, const float* loss, const int32_t* count_dev, aa_assistant* a,
                             float lr, int32_t thresh_mode, float threshold) {
     if (!ctx || !a) return AA_ERR_INVALID_ARG;

@@ -254,7 +254,8 @@ aa_status launch_batch_cut(aa_ctx_impl* c, const int32_t* idx, const int32_t* co
                            int32_t* out_consumed, int32_t* out_offsets, int64_t offsets_capacity);
 
 aa_status launch_instance_loss(aa_ctx_impl* c, const aa_logits& lg, const int32_t* labels, const int32_t* offsets,
-                               int64_t n_seg, const int32_t* count_dev, float* out_loss);
+                               int64_t n_seg, const int32_t* count_dev, float* out_loss, const int32_t* row_idx = nullptr,
+                               int64_t n_rows = 0);
 
 aa_status launch_assistant_step_dense(aa_ctx_impl* c, const DenseFeat& f, const int32_t* row_idx, int64_t n_stored,
                                       int64_t m_host, const int32_t* count_dev, const float* loss, float* w, float* b,

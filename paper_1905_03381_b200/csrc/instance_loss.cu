@@ -54,14 +54,16 @@ __global__ void __launch_bounds__(256) row_loss_group_kernel(LossParams p) {
         const int64_t r = group0 + it * groups_per_grid;
         RunState st = {-INFINITY, 0.0f};
         int y = -1;
+        int64_t src = -1;
         if (r < rows) {
-            y = checked_label(p, r);
-            if (y >= 0) scan_row<T>(st, static_cast<const T*>(p.logits) + r * p.row_stride, p.cols, gl, LPR);
+            src = source_row(p, r);
+            if (src >= 0) y = checked_label(p, src);
+            if (y >= 0) scan_row<T>(st, static_cast<const T*>(p.logits) + src * p.row_stride, p.cols, gl, LPR);
         }
         st = group_merge<LPR>(st);
         if (gl == 0 && r < rows) {
             float loss = 0.0f;
-            if (y >= 0) loss = finish_row(st, Vec<T>::one(static_cast<const T*>(p.logits) + r * p.row_stride + y));
+            if (y >= 0) loss = finish_row(st, Vec<T>::one(static_cast<const T*>(p.logits) + src * p.row_stride + y));
             p.out[r] = loss;
         }
     }
@@ -74,12 +76,13 @@ __global__ void __launch_bounds__(kRowThreads) row_loss_cta_kernel(LossParams p)
     const int64_t rows = effective_rows(p);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
-        const int y = checked_label(p, r);   // uniform over the CTA
+        const int64_t src = source_row(p, r);                 // uniform over the CTA
+        const int y = src >= 0 ? checked_label(p, src) : -1;
         if (y < 0) {
             if (threadIdx.x == 0) p.out[r] = 0.0f;
             continue;
         }
-        const T* row = static_cast<const T*>(p.logits) + r * p.row_stride;
+        const T* row = static_cast<const T*>(p.logits) + src * p.row_stride;
         RunState st = {-INFINITY, 0.0f};
         scan_row<T>(st, row, p.cols, threadIdx.x, kRowThreads);
         st = group_merge<32>(st);
@@ -154,24 +157,26 @@ aa_status launch_rows(aa_ctx_impl* c, LossParams& p) {
 }  // namespace
 
 aa_status launch_instance_loss(aa_ctx_impl* c, const aa_logits& lg, const int32_t* labels, const int32_t* offsets,
-                               int64_t n_seg, const int32_t* count_dev, float* out_loss) {
+                               int64_t n_seg, const int32_t* count_dev, float* out_loss, const int32_t* row_idx, int64_t n_rows) {
     LossParams p;
     p.logits = lg.data;
-    p.rows = lg.rows;
+    p.rows = row_idx ? n_rows : lg.rows;
+    p.row_idx = row_idx;
+    p.n_stored = lg.rows;
     p.cols = lg.cols;
     p.row_stride = lg.row_stride;
     p.labels = labels;
     p.count_dev = offsets ? nullptr : count_dev;
     p.ctl = c->ctl;
     p.out = offsets ? c->row_scratch : out_loss;
-    if (lg.rows > 0) {
-        aa_status st = launch_instance_loss_tma(c, p, lg.dtype);
+    if (p.rows > 0) {
+        aa_status st = row_idx ? AA_ERR_UNSUPPORTED : launch_instance_loss_tma(c, p, lg.dtype);   // the ring streams adjacent rows
         if (st == AA_ERR_UNSUPPORTED) st = lg.dtype == AA_BF16 ? launch_rows<uint16_t>(c, p) : launch_rows<float>(c, p);
         if (st != AA_OK) return st;
     }
     if (offsets && n_seg > 0) {
         const float* row_loss = c->row_scratch;
-        int64_t rows = lg.rows;
+        int64_t rows = p.rows;
         Control* ctl = c->ctl;
         void* args[] = {&row_loss, &offsets, &n_seg, &rows, &out_loss, &ctl};
         const int64_t want = (n_seg + 7) / 8;   // 8 warps per CTA

@@ -16,6 +16,8 @@ struct LossParams {
     int64_t rows, cols, row_stride;
     const int32_t* labels;
     const int32_t* count_dev;
+    const int32_t* row_idx;   // nullable: evaluated row k is stored row row_idx[k]; labels go by stored row
+    int64_t n_stored;         // stored rows (bounds the list entries)
     float* out;
     Control* ctl;
 };
@@ -90,6 +92,17 @@ __device__ __forceinline__ int64_t effective_rows(const LossParams& p) {
         rows = c < 0 ? 0 : (c < rows ? c : rows);
     }
     return rows;
+}
+
+// Stored row of evaluated row k: k itself, or the list entry (outside the stored rows: -1, latches AA_ERR_BAD_INDEX).
+__device__ __forceinline__ int64_t source_row(const LossParams& p, int64_t k) {
+    if (!p.row_idx) return k;
+    const int64_t r = __ldg(p.row_idx + k);
+    if ((unsigned long long)r >= (unsigned long long)p.n_stored) {
+        latch(p.ctl, AA_ERR_BAD_INDEX);
+        return -1;
+    }
+    return r;
 }
 
 // Label of row r: >= 0 valid; -1 padding or invalid (invalid latches AA_ERR_BAD_INDEX).

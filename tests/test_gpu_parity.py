@@ -515,3 +515,48 @@ def test_image_shape_full_pool(aa):
     # acceptance statistics over the whole pool from the GPU's own (verified) scores
     p_all = O.accept_prob(O.sigmoid(s.astype(np.float64)), cfg.gamma)
     assert abs(m - p_all.sum()) < 5 * math.sqrt((p_all * (1 - p_all)).sum())
+
+
+# --------------------------------------------------------------------------
+# losses of a batch list out of logits stored for the whole pool
+# --------------------------------------------------------------------------
+
+@pytest.mark.parametrize("rows,cols,dtype,m", [
+    (3000, 100, torch.float32, 1700), (517, 1000, torch.float32, 517), (300, 8200, torch.bfloat16, 120),
+    (64, 33000, torch.bfloat16, 40), (1, 5, torch.float32, 1),
+])
+def test_instance_loss_of_listed_rows(aa, rows, cols, dtype, m):
+    rng = np.random.default_rng(rows + cols)
+    lg = W.normal((rows, cols), 3.0, 41 + rows, dtype, DEV)
+    y = W.randint(0, cols, (rows,), 43 + rows, DEV).to(torch.int32)
+    y[rows // 2] = -1                                                   # a padding row: loss 0
+    listed = rng.integers(0, rows, m).astype(np.int32)                  # any order, repeats allowed
+    if m > 2:
+        listed[1] = rows // 2
+    idx = torch.from_numpy(listed).to(DEV)
+    out = torch.full((m + 3,), -5.0, dtype=torch.float32, device=DEV)
+    # the device count cuts the list short; entries at and beyond it stay untouched
+    m_dev = max(1, m - 2)
+    cnt = torch.tensor([m_dev], dtype=torch.int32, device=DEV)
+    aa.aa_instance_loss_rows(B.logits_desc(lg), y, idx, out, count_dev=cnt, n_rows=m)
+    torch.cuda.synchronize()
+    ref = O.instance_loss_rows(W.to_oracle(lg), y.cpu().numpy(), listed[:m_dev])
+    got = out.cpu().numpy()
+    assert np.all(np.abs(got[:m_dev] - ref) <= 1e-4)
+    if m_dev > 1 and m > 2:
+        assert got[1] == 0.0
+    assert np.all(got[m_dev:] == -5.0)
+
+
+def test_instance_loss_rows_bad_entry_latches_and_gives_zero():
+    ctx = B.AutoAssist(max_rows=1024, max_d=16, device=DEV)
+    lg = W.normal((100, 10), 1.0, 5, torch.float32, DEV)
+    y = torch.zeros(100, dtype=torch.int32, device=DEV)
+    idx = torch.tensor([3, 100, -1, 99], dtype=torch.int32, device=DEV)
+    out = torch.full((4,), -5.0, dtype=torch.float32, device=DEV)
+    ctx.aa_instance_loss_rows(B.logits_desc(lg), y, idx, out)
+    assert ctx.aa_device_status() == B.AA_ERR_BAD_INDEX
+    got = out.cpu().numpy()
+    assert got[1] == 0.0 and got[2] == 0.0 and got[0] > 0 and got[3] > 0
+    assert ctx.aa_device_status() == B.AA_OK
+    ctx.close()

@@ -612,3 +612,19 @@ def test_pipeline_schedule_lag_and_special_cases():
         other, _ = O.pipeline_linear_dense(pool_of, logits_of, w0, 0.05, 0.2, 77, 0.0, depth, steps)
         for t in range(steps):
             assert np.array_equal(base[t]["B"], other[t]["B"]) and np.array_equal(other[t]["w"], w0)
+
+
+def test_instance_loss_rows_is_the_row_loss_of_the_listed_rows():
+    """Brute force with scipy's logsumexp on the listed rows; the identity list gives the plain per-row losses;
+    a repeated entry repeats its loss."""
+    from scipy.special import logsumexp
+
+    rng = np.random.default_rng(17)
+    lg = (rng.normal(size=(50, 9)) * 3).astype(np.float32)
+    y = rng.integers(0, 9, 50).astype(np.int32)
+    rows = np.array([49, 0, 7, 7, 23, 1], np.int32)
+    got = O.instance_loss_rows(lg, y, rows)
+    want = [logsumexp(lg[r].astype(np.float64)) - float(lg[r, y[r]]) for r in rows]
+    assert np.allclose(got, want, rtol=1e-12, atol=1e-12)
+    assert got[2] == got[3]
+    assert np.array_equal(O.instance_loss_rows(lg, y, np.arange(50)), O.row_loss(lg, y))
