@@ -172,6 +172,7 @@ __global__ void __launch_bounds__(256) linear_apply_kernel(StepParams p, int par
 }
 
 // ---------------------------------------------------------------- CSR
+constexpr int kCsrStepUnroll = 8;
 template <int LPR>
 __global__ void __launch_bounds__(256) csr_residual_kernel(StepParams p) {
     __shared__ double red[8];
@@ -188,10 +189,27 @@ __global__ void __launch_bounds__(256) csr_residual_kernel(StepParams p) {
         float acc = 0.0f;
         if (r >= 0) {
             const int e0 = __ldg(p.csr.indptr + r), e1 = __ldg(p.csr.indptr + r + 1);
-            for (int e = e0 + gl; e < e1; e += LPR) {
-                const int c = __ldg(p.csr.col + e);
-                if ((unsigned long long)(unsigned int)c < (unsigned long long)p.csr.d) acc = fmaf(__ldg(p.csr.val + e), p.w[c], acc);
-                else latch(p.ctl, AA_ERR_BAD_INDEX);
+            // kCsrStepUnroll entries per lane and trip: their loads, then their weight gathers, are in flight together
+            for (int e = e0 + gl; e < e1; e += kCsrStepUnroll * LPR) {
+                int c[kCsrStepUnroll];
+                float v[kCsrStepUnroll], wq[kCsrStepUnroll];
+#pragma unroll
+                for (int u = 0; u < kCsrStepUnroll; ++u) {
+                    const int ee = e + u * LPR;
+                    const bool in = ee < e1;
+                    c[u] = in ? __ldg(p.csr.col + ee) : 0;
+                    v[u] = in ? __ldg(p.csr.val + ee) : 0.0f;
+                }
+                bool bad = false;
+#pragma unroll
+                for (int u = 0; u < kCsrStepUnroll; ++u) {
+                    const bool ok = (unsigned long long)(unsigned int)c[u] < (unsigned long long)p.csr.d;
+                    bad |= !ok;
+                    wq[u] = ok ? p.w[c[u]] : 0.0f;
+                }
+#pragma unroll
+                for (int u = 0; u < kCsrStepUnroll; ++u) acc = fmaf(v[u], wq[u], acc);
+                if (bad) latch(p.ctl, AA_ERR_BAD_INDEX);
             }
         }
 #pragma unroll
@@ -229,9 +247,19 @@ __global__ void __launch_bounds__(256) csr_scatter_kernel(StepParams p) {
         const float step = scale * p.residual[i];
         if (gl == 0) bias_acc += step;
         const int e0 = __ldg(p.csr.indptr + r), e1 = __ldg(p.csr.indptr + r + 1);
-        for (int e = e0 + gl; e < e1; e += LPR) {
-            const int c = __ldg(p.csr.col + e);
-            if ((unsigned long long)(unsigned int)c < (unsigned long long)p.csr.d) atomicAdd(w_dst + c, step * __ldg(p.csr.val + e));
+        for (int e = e0 + gl; e < e1; e += kCsrStepUnroll * LPR) {
+            int c[kCsrStepUnroll];
+            float v[kCsrStepUnroll];
+#pragma unroll
+            for (int u = 0; u < kCsrStepUnroll; ++u) {
+                const int ee = e + u * LPR;
+                const bool in = ee < e1;
+                c[u] = in ? __ldg(p.csr.col + ee) : -1;
+                v[u] = in ? __ldg(p.csr.val + ee) : 0.0f;
+            }
+#pragma unroll
+            for (int u = 0; u < kCsrStepUnroll; ++u)
+                if ((unsigned long long)(unsigned int)c[u] < (unsigned long long)p.csr.d) atomicAdd(w_dst + c[u], step * v[u]);
         }
     }
 #pragma unroll
@@ -363,8 +391,8 @@ aa_status launch_assistant_step_csr(aa_ctx_impl* c, const CsrFeat& f, const int3
         if (f.d + 1 > c->partial_floats) return AA_ERR_WORKSPACE;
         if (cudaMemsetAsync(c->partials, 0, sizeof(float) * (size_t)(f.d + 1), c->stream) != cudaSuccess) return AA_ERR_CUDA;
     }
-    int lpr = 4;
-    while (lpr < 32 && lpr * 4 <= f.mean_nnz) lpr <<= 1;
+    int lpr = 4;   // about one unrolled trip per lane for a row of average length
+    while (lpr < 32 && (float)lpr * kCsrStepUnroll * 1.1f < f.mean_nnz) lpr <<= 1;
     const int64_t rows_per_cta = 256 / lpr;
     const int64_t want = (m_host + rows_per_cta - 1) / rows_per_cta;
     const int cap = c->sm_count * 8;

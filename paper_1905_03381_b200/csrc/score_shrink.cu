@@ -138,6 +138,7 @@ __global__ void __launch_bounds__(kScanThreads) score_shrink_dense_kernel(DenseF
 }
 
 // ---------------------------------------------------------------- CSR bag-of-words Assistant
+constexpr int kCsrUnroll = 8;
 template <int LPR>
 __global__ void __launch_bounds__(kScanThreads) score_shrink_csr_kernel(CsrFeat f, ShrinkParams p) {
     __shared__ TailSmem sm;
@@ -156,10 +157,29 @@ __global__ void __launch_bounds__(kScanThreads) score_shrink_csr_kernel(CsrFeat 
             float acc = 0.0f;
             if (r >= 0) {
                 const int e0 = __ldg(f.indptr + r), e1 = __ldg(f.indptr + r + 1);
-                for (int e = e0 + gl; e < e1; e += LPR) {
-                    const int c = __ldg(f.col + e);
-                    if ((unsigned long long)(unsigned int)c < (unsigned long long)f.d) acc = fmaf(__ldg(f.val + e), __ldg(f.w + c), acc);
-                    else latch(p.ctl, AA_ERR_BAD_INDEX);
+                // kCsrUnroll entries per lane and trip: their column/value loads, then their weight gathers, are in
+                // flight together (the row is a chain of three dependent memory round trips, not one per entry)
+                for (int e = e0 + gl; e < e1; e += kCsrUnroll * LPR) {
+                    int c[kCsrUnroll];
+                    float v[kCsrUnroll];
+#pragma unroll
+                    for (int u = 0; u < kCsrUnroll; ++u) {
+                        const int ee = e + u * LPR;
+                        const bool in = ee < e1;
+                        c[u] = in ? __ldg(f.col + ee) : 0;
+                        v[u] = in ? __ldg(f.val + ee) : 0.0f;
+                    }
+                    float wq[kCsrUnroll];
+                    bool bad = false;
+#pragma unroll
+                    for (int u = 0; u < kCsrUnroll; ++u) {
+                        const bool ok = (unsigned long long)(unsigned int)c[u] < (unsigned long long)f.d;
+                        bad |= !ok;
+                        wq[u] = ok ? __ldg(f.w + c[u]) : 0.0f;
+                    }
+#pragma unroll
+                    for (int u = 0; u < kCsrUnroll; ++u) acc = fmaf(v[u], wq[u], acc);
+                    if (bad) latch(p.ctl, AA_ERR_BAD_INDEX);
                 }
             }
 #pragma unroll
@@ -278,7 +298,9 @@ aa_status launch_score_shrink_dense(aa_ctx_impl* c, const DenseFeat& f_in, Shrin
 
 aa_status launch_score_shrink_csr(aa_ctx_impl* c, const CsrFeat& f_in, ShrinkParams sp) {
     CsrFeat f = f_in;
-    int lpr = pow2_ceil((int64_t)(f.mean_nnz / 4.0f + 0.5f));
+    // about one unrolled trip per lane for a row of average length
+    int lpr = pow2_ceil((int64_t)(f.mean_nnz / kCsrUnroll + 0.5f));
+    if (lpr > 4 && (float)(lpr / 2) * kCsrUnroll * 1.1f >= f.mean_nnz) lpr >>= 1;
     lpr = lpr < 4 ? 4 : (lpr > 32 ? 32 : lpr);
     aa_status st = finish_shrink_params(c, sp, choose_tile_rows(c, sp.n_cand, 8.0 * f.mean_nnz + 4.0, 64.0 * 1024));
     if (st != AA_OK) return st;
