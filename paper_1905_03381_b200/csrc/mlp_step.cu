@@ -412,30 +412,80 @@ mlp_w1_grad_kernel(const __grid_constant__ CUtensorMap map_pt, const __grid_cons
 __global__ void __launch_bounds__(256) mlp_apply_w1_kernel(MlpStepParams p) {
     const int64_t m = mlp_batch_size(p);
     if (m <= 0) return;
-    const int64_t total = (int64_t)p.g.hidden * p.d;
     const float scale = p.lr / (float)m;
+    const float inv_m = 1.0f / (float)m;
+    if ((p.d & 3) == 0 && (p.d_pad & 3) == 0 && (((uintptr_t)p.W1 | (uintptr_t)p.part) & 15) == 0 && ((uintptr_t)p.W1_bf16 & 7) == 0) {
+        // four adjacent feature columns per thread: 16-byte loads of the split-K partials and of W1
+        const int64_t dq = p.d >> 2, total = (int64_t)p.g.hidden * dq;
+        for (int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; q < total; q += (int64_t)gridDim.x * blockDim.x) {
+            const int64_t u = q / dq, k = (q - u * dq) << 2;
+            float4 g = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+#pragma unroll 4
+            for (int s = 0; s < p.splits; ++s) {
+                const float4 t = __ldcs(reinterpret_cast<const float4*>(p.part + ((int64_t)s * p.g.hidden + u) * p.d_pad + k));
+                g.x += t.x; g.y += t.y; g.z += t.z; g.w += t.w;
+            }
+            const float w2u = __ldg(p.w2 + u);
+            float4* wp = reinterpret_cast<float4*>(p.W1 + u * p.d + k);
+            float4 w = *wp;
+            const float gv[4] = {g.x, g.y, g.z, g.w};
+            float wv[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                wv[e] = p.adam.on ? adam_update(p.adam, wv[e], w2u * gv[e] * inv_m, p.lr, u * p.d + k + e) : wv[e] - scale * w2u * gv[e];
+            *wp = make_float4(wv[0], wv[1], wv[2], wv[3]);
+            __nv_bfloat162 lo = __floats2bfloat162_rn(wv[0], wv[1]), hi = __floats2bfloat162_rn(wv[2], wv[3]);
+            uint2 packed;
+            packed.x = *reinterpret_cast<uint32_t*>(&lo);
+            packed.y = *reinterpret_cast<uint32_t*>(&hi);
+            *reinterpret_cast<uint2*>(p.W1_bf16 + u * p.d + k) = packed;
+        }
+        return;
+    }
+    const int64_t total = (int64_t)p.g.hidden * p.d;
     for (int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; q < total; q += (int64_t)gridDim.x * blockDim.x) {
         const int64_t u = q / p.d, k = q - u * p.d;
         float g = 0.0f;
         for (int s = 0; s < p.splits; ++s) g += p.part[((int64_t)s * p.g.hidden + u) * p.d_pad + k];
-        const float w = p.adam.on ? adam_update(p.adam, p.W1[q], __ldg(p.w2 + u) * g / (float)m, p.lr, q)
+        const float w = p.adam.on ? adam_update(p.adam, p.W1[q], __ldg(p.w2 + u) * g * inv_m, p.lr, q)
                                   : p.W1[q] - scale * __ldg(p.w2 + u) * g;
         p.W1[q] = w;
         p.W1_bf16[q] = __float2bfloat16_rn(w);
     }
 }
 
-__global__ void __launch_bounds__(kMaxHidden) mlp_apply_small_kernel(MlpStepParams p, int ctas) {
+// b1, w2, b2 from the per-CTA column sums: kSmallSlices thread rows share the CTAs (loads in flight together), the
+// slices are added in a fixed order.
+constexpr int kSmallSlices = 4;
+__global__ void __launch_bounds__(kMaxHidden * kSmallSlices) mlp_apply_small_kernel(MlpStepParams p, int ctas) {
+    __shared__ float part_w2[kSmallSlices][kMaxHidden], part_b1[kSmallSlices][kMaxHidden], part_b2[32];
     const int64_t m = mlp_batch_size(p);
     if (m <= 0) return;
     const float scale = p.lr / (float)m;
-    const int u = threadIdx.x;
-    if (u < p.g.hidden) {
+    const int u = threadIdx.x % kMaxHidden, slice = threadIdx.x / kMaxHidden;
+    {
         float g_w2 = 0.0f, g_b1 = 0.0f;
-        for (int c = 0; c < ctas; ++c) {
+#pragma unroll 8
+        for (int c = slice; c < ctas; c += kSmallSlices) {
             const float* in = p.small + (int64_t)c * (2 * kMaxHidden + 1);
             g_w2 += in[u];
             g_b1 += in[kMaxHidden + u];
+        }
+        part_w2[slice][u] = g_w2;
+        part_b1[slice][u] = g_b1;
+    }
+    if (threadIdx.x < 32) {
+        float g_b2 = 0.0f;
+        for (int c = threadIdx.x; c < ctas; c += 32) g_b2 += p.small[(int64_t)c * (2 * kMaxHidden + 1) + 2 * kMaxHidden];
+        part_b2[threadIdx.x] = g_b2;
+    }
+    __syncthreads();
+    if (slice == 0 && u < p.g.hidden) {
+        float g_w2 = 0.0f, g_b1 = 0.0f;
+#pragma unroll
+        for (int q = 0; q < kSmallSlices; ++q) {
+            g_w2 += part_w2[q][u];
+            g_b1 += part_b1[q][u];
         }
         const float w2_old = p.w2[u];
         const int64_t hd = (int64_t)p.g.hidden * p.d;      // moments: W1, then b1, w2, b2
@@ -447,9 +497,9 @@ __global__ void __launch_bounds__(kMaxHidden) mlp_apply_small_kernel(MlpStepPara
             p.w2[u] = w2_old - scale * g_w2;
         }
     }
-    if (u == 0) {
+    if (threadIdx.x == 0) {
         float g_b2 = 0.0f;
-        for (int c = 0; c < ctas; ++c) g_b2 += p.small[(int64_t)c * (2 * kMaxHidden + 1) + 2 * kMaxHidden];
+        for (int q = 0; q < 32; ++q) g_b2 += part_b2[q];
         p.b2[0] = p.adam.on ? adam_update(p.adam, p.b2[0], g_b2 / (float)m, p.lr, (int64_t)p.g.hidden * p.d + 2 * p.g.hidden)
                             : p.b2[0] - scale * g_b2;
     }
@@ -541,12 +591,13 @@ aa_status launch_assistant_step_mlp(aa_ctx_impl* c, const MlpFeat& f, float* W1_
         // 3. updates (W1 first: it reads the old w2)
         void* args3[] = {&p};
         const int64_t total = f.hidden * f.d;
-        int agrid = (int)((total + 255) / 256);
+        int agrid = (int)((total / 4 + 255) / 256);
         if (agrid > c->sm_count * 8) agrid = c->sm_count * 8;
+        if (agrid < 1) agrid = 1;
         if (cudaLaunchKernel((const void*)mlp_apply_w1_kernel, dim3(agrid), dim3(256), args3, 0, c->stream) != cudaSuccess) return AA_ERR_CUDA;
         ++c->launches;
         void* args4[] = {&p, &grid};
-        if (cudaLaunchKernel((const void*)mlp_apply_small_kernel, dim3(1), dim3(kMaxHidden), args4, 0, c->stream) != cudaSuccess)
+        if (cudaLaunchKernel((const void*)mlp_apply_small_kernel, dim3(1), dim3(kMaxHidden * kSmallSlices), args4, 0, c->stream) != cudaSuccess)
             return AA_ERR_CUDA;
         ++c->launches;
     }
