@@ -5,7 +5,7 @@
 //   producer warp : per 64-wide K-slice, 256 feature rows x 64 columns and `hidden` W1 rows x 64
 //                   columns (128-byte swizzle) into a 3-stage ring.  Rows come as one TMA box
 //                   when the tile's rows are adjacent in memory, or as 64 four-row gathers
-//                   (tile::gather4, two per lane) when a row list selects them.
+//                   (tile::gather4, spread over eight warps) when a row list selects them.
 //   MMA warp      : tcgen05.mma M = 128, N = hidden, K = 16, eight per stage; commits every
 //                   stage back to the producer and every finished super-tile to `acc_full`.
 // The consumer of the accumulators arrives `acc_consumers` times on `acc_empty` per super-tile.
@@ -23,7 +23,7 @@ constexpr int kMlpStages = 3;
 constexpr int kABytes = kSuperRows * 128;       // feature slice of one stage
 constexpr int kMaxHidden = 256;
 constexpr int kTmemCols = 512;
-constexpr int kGatherWarps = 4;                 // warps that issue the row gathers when a row list selects the rows
+constexpr int kGatherWarps = 8;                 // warps that issue the row gathers when a row list selects the rows
 
 struct MlpGeom {
     int hidden;
@@ -79,8 +79,8 @@ template <bool GATHER>
 __device__ __forceinline__ bool mlp_produce(TilePipe* tp, unsigned char* ring, const CUtensorMap* map_x, const CUtensorMap* map_w,
                                             const MlpGeom& g, unsigned int n_tiles, const int32_t* rows, long long n_list,
                                             long long n_stored, int part = 0) {
-    // Gathered rows are fetched by kGatherWarps warps (part = 0 .. kGatherWarps - 1), 64 rows each, one four-row
-    // gather per lane and stage: the gathers a single warp issues retire at only about one per 43 ns.  Part 0 is the
+    // Gathered rows are fetched by kGatherWarps warps (part = 0 .. kGatherWarps - 1), 32 rows each, one four-row
+    // gather per issuing lane and stage: the gathers a single warp issues retire at only about one per 43 ns.  Part 0 is the
     // producer proper (it also posts the expected bytes and loads W1); the others follow the same barriers.
     const int lane = threadIdx.x & 31;
     const bool helper = part != 0;

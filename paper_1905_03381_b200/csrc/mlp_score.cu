@@ -27,7 +27,8 @@ namespace aa {
 
 namespace {
 
-constexpr int kMlpThreads = 448;               // warps 12, 13 only help with row gathers
+constexpr int kMlpThreads = 576;               // with a candidate list: warps 12..17 only help with row gathers
+constexpr int kMlpThreadsDense = 384;          // adjacent rows: one box per stage, no helpers
 constexpr int kEpiWarps = 8;
 
 struct ScoreControl {
@@ -48,7 +49,7 @@ __device__ __forceinline__ void mlp_give_up(const ShrinkParams& p, TilePipe* tp)
 }
 
 template <bool GATHER>
-__global__ void __launch_bounds__(kMlpThreads, 1)
+__global__ void __launch_bounds__(GATHER ? kMlpThreads : kMlpThreadsDense, 1)
 mlp_score_shrink_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                         MlpKernelParams mp, ShrinkParams p) {
     extern __shared__ unsigned char smem_raw[];
@@ -70,7 +71,7 @@ mlp_score_shrink_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
         prefetch_tensormap(&map_x);
         prefetch_tensormap(&map_w);
     }
-    for (int j = tid; j < kMaxHidden; j += kMlpThreads) {
+    for (int j = tid; j < kMaxHidden; j += (int)blockDim.x) {
         b1_s[j] = j < mp.g.hidden ? mp.b1[j] : 0.0f;
         w2_s[j] = j < mp.g.hidden ? mp.w2[j] : 0.0f;
     }
@@ -209,7 +210,7 @@ aa_status launch_score_shrink_mlp(aa_ctx_impl* c, const MlpFeat& f, ShrinkParams
     int grid = c->sm_count;
     if ((unsigned int)grid > sp.n_tiles) grid = (int)sp.n_tiles;
     void* args[] = {&map_x, &map_w, &mp, &sp};
-    if (cudaLaunchKernel(kernel, dim3(grid), dim3(kMlpThreads), args, smem, c->stream) != cudaSuccess) return AA_ERR_CUDA;
+    if (cudaLaunchKernel(kernel, dim3(grid), dim3(gather ? kMlpThreads : kMlpThreadsDense), args, smem, c->stream) != cudaSuccess) return AA_ERR_CUDA;
     ++c->launches;
     return AA_OK;
 }

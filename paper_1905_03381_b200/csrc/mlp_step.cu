@@ -27,7 +27,7 @@ namespace aa {
 
 namespace {
 
-constexpr int kStepMlpThreads = 448;          // warps 12, 13 only help with row gathers
+constexpr int kStepMlpThreads = 576;          // warps 12..17 only help with row gathers
 constexpr int kStepEpiWarps = 8;
 constexpr int kMaxMlpCtas = 192;              // bound on the grids below (workspace sizing)
 constexpr int kFeatChunk = 256;               // feature columns per CTA of the W1-gradient kernel
@@ -294,21 +294,22 @@ mlp_w1_grad_kernel(const __grid_constant__ CUtensorMap map_pt, const __grid_cons
     if (n_q > 4) n_q = 4;
 
     if (warp == 0 || (GATHER && (warp == 3 || warp >= 12))) {
-        // ------------------------------------------------------------ producer (warp 0) and, for gathered rows, three helpers:
-        // gather warp q fetches 64-column chunk q of every stage, sixteen four-row gathers (one per lane); warp 0 also posts
-        // the expected bytes and loads the P^T box.
+        // ------------------------------------------------------------ producer (warp 0) and, for gathered rows, seven helpers:
+        // gather warp q fetches rows (q & 1) * 32 .. + 32 of 64-column chunk q >> 1 of every stage, eight four-row gathers
+        // (one per issuing lane); warp 0 also posts the expected bytes and loads the P^T box.
         const int part = warp == 0 ? 0 : (warp == 3 ? 1 : warp - 10);
+        const int chunk_q = part >> 1, half = part & 1;
         int stage = 0, j = 0;
         uint32_t phase = 0;
         bool ok = true;
         for (int sl = 0; sl < n_slices; ++sl) {
             const int64_t i0 = (s_begin + sl) * kRowSlice;
             int r0 = 0, r1 = 0, r2 = 0, r3 = 0;
-            if (GATHER && lane < 16) {
+            if (GATHER && lane < 8) {
                 int rr[4];
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    const int64_t i = i0 + lane * 4 + q;
+                    const int64_t i = i0 + half * 32 + lane * 4 + q;
                     long long row = i < m ? (long long)p.row_idx[i] : 0;
                     if ((unsigned long long)row >= (unsigned long long)p.n_stored) row = 0;   // its P column is zero
                     rr[q] = (int)row;
@@ -326,8 +327,9 @@ mlp_w1_grad_kernel(const __grid_constant__ CUtensorMap map_pt, const __grid_cons
             }
             if (GATHER) {
                 __syncwarp();
-                if (lane < 16 && part < n_q)
-                    tma_gather4(x_dst + part * kXChunkBytes + (lane * 4) * 128, &map_x, col0 + part * 64, r0, r1, r2, r3, &gp->full[stage]);
+                if (lane < 8 && chunk_q < n_q)
+                    tma_gather4(x_dst + chunk_q * kXChunkBytes + (half * 32 + lane * 4) * 128, &map_x, col0 + chunk_q * 64, r0, r1, r2, r3,
+                                &gp->full[stage]);
             }
             __syncwarp();
             ++j;
