@@ -20,6 +20,9 @@ namespace aa {
 constexpr int kSuperRows = 256;                 // rows per super-tile (two M = 128 accumulators)
 constexpr int kSliceK = 64;                     // bf16 elements per 128-byte swizzled row
 constexpr int kMlpStages = 3;
+constexpr int kMaxMlpStages = 4;
+constexpr int kHalfRows = 128;                  // rows per tile when two accumulators alternate (one M = 128 accumulator each)
+constexpr int kHalfStages = 4;
 constexpr int kABytes = kSuperRows * 128;       // feature slice of one stage
 constexpr int kMaxHidden = 256;
 constexpr int kTmemCols = 512;
@@ -33,18 +36,18 @@ struct MlpGeom {
 };
 
 struct TilePipe {
-    uint64_t full[kMlpStages], empty[kMlpStages];
-    uint64_t acc_full, acc_empty, drain;
+    uint64_t full[kMaxMlpStages], empty[kMaxMlpStages];
+    uint64_t acc_full[2], acc_empty[2], drain;   // 256-row super-tiles use entry 0; 128-row tiles alternate between the two
     uint32_t tmem_base;
     int abort_flag;
 };
 
-inline MlpGeom make_mlp_geom(int64_t d, int64_t hidden) {
+inline MlpGeom make_mlp_geom(int64_t d, int64_t hidden, int tile_rows = kSuperRows) {
     MlpGeom g;
     g.hidden = (int)hidden;
     g.k_slices = (int)((d + kSliceK - 1) / kSliceK);
     g.b_bytes = (uint32_t)hidden * 128u;
-    g.stage_bytes = ((uint32_t)kABytes + g.b_bytes + 1023u) & ~1023u;
+    g.stage_bytes = ((uint32_t)tile_rows * 128u + g.b_bytes + 1023u) & ~1023u;
     return g;
 }
 
@@ -61,21 +64,23 @@ __device__ __forceinline__ void tma_gather4(void* dst, const CUtensorMap* map, i
 }
 
 __device__ __forceinline__ void tile_pipe_init(TilePipe* tp, uint32_t acc_consumers) {
-    for (int s = 0; s < kMlpStages; ++s) {
+    for (int s = 0; s < kMaxMlpStages; ++s) {
         mbar_init(&tp->full[s], 1);
         mbar_init(&tp->empty[s], 1);
     }
-    mbar_init(&tp->acc_full, 1);
-    mbar_init(&tp->acc_empty, acc_consumers);
+    for (int b = 0; b < 2; ++b) {
+        mbar_init(&tp->acc_full[b], 1);
+        mbar_init(&tp->acc_empty[b], acc_consumers);
+    }
     mbar_init(&tp->drain, 1);
     tp->abort_flag = 0;
 }
 
-// Whole warp.  Tiles blockIdx.x, blockIdx.x + gridDim.x, ... below n_tiles.  rows: nullptr = tile t
-// holds stored rows [256 t, 256 t + 256); otherwise row k of the list (k < n_list) names the
+// Whole warp.  Tiles of ROWS rows: blockIdx.x, blockIdx.x + gridDim.x, ... below n_tiles.  rows: nullptr = tile t
+// holds stored rows [ROWS t, ROWS t + ROWS) (the feature map's box is ROWS rows high); otherwise row k of the list (k < n_list) names the
 // stored row, entries outside [0, n_stored) or past the list read row 0 (their results are
 // discarded by the consumer).  Returns false if a wait gave up.
-template <bool GATHER>
+template <bool GATHER, int ROWS = kSuperRows, int STAGES = kMlpStages>
 __device__ __forceinline__ bool mlp_produce(TilePipe* tp, unsigned char* ring, const CUtensorMap* map_x, const CUtensorMap* map_w,
                                             const MlpGeom& g, unsigned int n_tiles, const int32_t* rows, long long n_list,
                                             long long n_stored, int part = 0) {
@@ -88,10 +93,11 @@ __device__ __forceinline__ bool mlp_produce(TilePipe* tp, unsigned char* ring, c
     int stage = 0, j = 0;
     uint32_t phase = 0;
     bool ok = true;
-    constexpr int kRowsPerPart = kSuperRows / kGatherWarps;
+    constexpr int kRowsPerPart = ROWS / kGatherWarps;
+    constexpr uint32_t kTileBytes = (uint32_t)ROWS * 128u;
     const bool gather_lane = lane < kRowsPerPart / 4;
     for (unsigned int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-        const long long k0 = (long long)tile * kSuperRows;
+        const long long k0 = (long long)tile * ROWS;
         int r[4] = {0, 0, 0, 0};
         if (GATHER && gather_lane) {
 #pragma unroll
@@ -106,8 +112,8 @@ __device__ __forceinline__ bool mlp_produce(TilePipe* tp, unsigned char* ring, c
             if (!mbar_wait(&tp->empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
             unsigned char* a_dst = ring + (size_t)stage * g.stage_bytes;
             if (lane == 0 && !helper) {
-                mbar_arrive_expect_tx(&tp->full[stage], (uint32_t)kABytes + g.b_bytes);
-                tma_load_2d(a_dst + kABytes, map_w, ks * kSliceK, 0, &tp->full[stage]);
+                mbar_arrive_expect_tx(&tp->full[stage], kTileBytes + g.b_bytes);
+                tma_load_2d(a_dst + kTileBytes, map_w, ks * kSliceK, 0, &tp->full[stage]);
                 if (!GATHER) tma_load_2d(a_dst, map_x, ks * kSliceK, (int)k0, &tp->full[stage]);
             }
             if (GATHER) {
@@ -117,14 +123,14 @@ __device__ __forceinline__ bool mlp_produce(TilePipe* tp, unsigned char* ring, c
             }
             __syncwarp();
             ++j;
-            if (++stage == kMlpStages) { stage = 0; phase ^= 1u; }
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
     }
     if (!ok) {
         // let copies still in flight land before the CTA's shared memory goes away
-        const int pending = j < kMlpStages ? j : kMlpStages;
+        const int pending = j < STAGES ? j : STAGES;
         for (int back = 1; back <= pending; ++back) {
-            const int jj = j - back, st = jj % kMlpStages, use = jj / kMlpStages;
+            const int jj = j - back, st = jj % STAGES, use = jj / STAGES;
             const long long t0 = clock64();
             while (!mbar_try_wait(&tp->full[st], (uint32_t)(use & 1)) && clock64() - t0 < kWaitCycles) {}
         }
@@ -133,35 +139,44 @@ __device__ __forceinline__ bool mlp_produce(TilePipe* tp, unsigned char* ring, c
 }
 
 // Whole warp; lane 0 issues.  Returns false if a wait gave up.  On return every MMA issued here has retired.
+// ROWS = 256: both accumulators hold one super-tile (the consumer drains them before the next one starts).
+// ROWS = 128: tile `it` of this CTA accumulates into accumulator it & 1, so the consumer of one tile overlaps
+// the products of the next.
+template <int ROWS = kSuperRows, int STAGES = kMlpStages>
 __device__ __forceinline__ bool mlp_issue_mma(TilePipe* tp, unsigned char* ring, const MlpGeom& g, unsigned int n_tiles, uint32_t tmem_base) {
     const int lane = threadIdx.x & 31;
     volatile int* abort_flag = &tp->abort_flag;
     const uint32_t idesc = umma_idesc_bf16(128, g.hidden, false, false);
+    constexpr uint32_t kTileBytes = (uint32_t)ROWS * 128u;
     int stage = 0, it = 0;
     uint32_t phase = 0;
     bool ok = true;
     for (unsigned int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
-        // the consumer has drained both accumulators of the previous super-tile
-        if (!mbar_wait(&tp->acc_empty, (uint32_t)((it & 1) ^ 1), abort_flag)) { ok = false; break; }
+        // the consumer has drained the accumulator(s) this tile writes
+        const int buf = ROWS == kSuperRows ? 0 : (it & 1);
+        const int use = ROWS == kSuperRows ? it : (it >> 1);
+        if (!mbar_wait(&tp->acc_empty[buf], (uint32_t)((use & 1) ^ 1), abort_flag)) { ok = false; break; }
         tc_fence_after_sync();
+        const uint32_t acc_addr = tmem_base + (uint32_t)(buf * kMaxHidden);
         for (int ks = 0; ks < g.k_slices; ++ks) {
             if (!mbar_wait(&tp->full[stage], phase, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
             if (lane == 0) {
                 const uint32_t a_addr = smem_u32(ring + (size_t)stage * g.stage_bytes);
-                const uint32_t b_addr = a_addr + kABytes;
+                const uint32_t b_addr = a_addr + kTileBytes;
 #pragma unroll
                 for (int k = 0; k < kSliceK / 16; ++k) {
                     const uint64_t b_desc = umma_smem_desc(b_addr + k * 32, 16, 1024);
                     const bool acc = (ks | k) != 0;
-                    umma_bf16(tmem_base, umma_smem_desc(a_addr + k * 32, 16, 1024), b_desc, idesc, acc);
-                    umma_bf16(tmem_base + kMaxHidden, umma_smem_desc(a_addr + 128 * 128 + k * 32, 16, 1024), b_desc, idesc, acc);
+                    umma_bf16(acc_addr, umma_smem_desc(a_addr + k * 32, 16, 1024), b_desc, idesc, acc);
+                    if (ROWS == kSuperRows)
+                        umma_bf16(acc_addr + kMaxHidden, umma_smem_desc(a_addr + 128 * 128 + k * 32, 16, 1024), b_desc, idesc, acc);
                 }
-                umma_commit(&tp->empty[stage]);                            // stage reusable once these MMAs are done
-                if (ks == g.k_slices - 1) umma_commit(&tp->acc_full);      // super-tile finished
+                umma_commit(&tp->empty[stage]);                                 // stage reusable once these MMAs are done
+                if (ks == g.k_slices - 1) umma_commit(&tp->acc_full[buf]);      // tile finished
             }
             __syncwarp();
-            if (++stage == kMlpStages) { stage = 0; phase ^= 1u; }
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
     }
     if (lane == 0) umma_commit(&tp->drain);

@@ -126,7 +126,7 @@ mlp_score_shrink_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
         int it = 0;
         for (unsigned int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
             const int buf = it & 1;
-            if (!mbar_wait(&tp->acc_full, (uint32_t)(it & 1), abort_flag) ||
+            if (!mbar_wait(&tp->acc_full[0], (uint32_t)(it & 1), abort_flag) ||
                 !mbar_wait(&cb->s_empty[buf], (uint32_t)(((it >> 1) & 1) ^ 1), abort_flag)) {
                 if (lane == 0) mlp_give_up(p, tp);
                 break;
@@ -151,7 +151,7 @@ mlp_score_shrink_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(&tp->acc_empty);
+                mbar_arrive(&tp->acc_empty[0]);
                 mbar_arrive(&cb->s_full[buf]);
             }
         }

@@ -3,7 +3,9 @@
 // back-propagated through both layers on the tcgen05 tensor cores.
 //
 //   mlp_residual_kernel  forward pass over the batch rows under the current parameters (same
-//                        TMA/MMA pipeline as scoring), then per row  z = 1[loss > T],
+//                        TMA/MMA pipeline as scoring, but in tiles of 128 rows whose two
+//                        accumulators alternate: the passes over one tile's accumulator run
+//                        while the products of the next tile are issued), then per row  z = 1[loss > T],
 //                        r = sigmoid(s) - z,  and per hidden unit u the factor
 //                        P[i][u] = r_i [a_iu > 0]  of delta1_iu = r_i w2_u [a_iu > 0].
 //                        P is stored transposed in bf16 ([hidden x rows]); the column sums
@@ -28,7 +30,7 @@ namespace aa {
 namespace {
 
 constexpr int kStepMlpThreads = 576;          // warps 12..17 only help with row gathers
-constexpr int kStepEpiWarps = 8;
+constexpr int kStepEpiWarps = 8;              // two sets of four: set b drains accumulator b
 constexpr int kMaxMlpCtas = 192;              // bound on the grids below (workspace sizing)
 constexpr int kFeatChunk = 256;               // feature columns per CTA of the W1-gradient kernel
 constexpr int kRowSlice = 64;                 // batch rows per K-slice of the W1-gradient kernel
@@ -97,7 +99,7 @@ __global__ void __launch_bounds__(kStepMlpThreads, 1)
 mlp_residual_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, MlpStepParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* ring = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    float* b1_s = reinterpret_cast<float*>(ring + (size_t)kMlpStages * p.g.stage_bytes);
+    float* b1_s = reinterpret_cast<float*>(ring + (size_t)kHalfStages * p.g.stage_bytes);
     float* w2_s = b1_s + kMaxHidden;
     float* col_s = w2_s + kMaxHidden;                        // [kStepEpiWarps][2][kMaxHidden] column sums per warp
     double* red = reinterpret_cast<double*>(col_s + kStepEpiWarps * 2 * kMaxHidden);   // [warps]
@@ -107,7 +109,7 @@ mlp_residual_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int hidden = p.g.hidden;
     if (tid == 0) {
-        tile_pipe_init(tp, kStepEpiWarps);
+        tile_pipe_init(tp, kStepEpiWarps / 2);
         mbar_fence_init();
         prefetch_tensormap(&map_x);
         prefetch_tensormap(&map_w);
@@ -137,34 +139,35 @@ mlp_residual_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
         T_shrink = m > 0 ? total / (double)m : 0.0;
     }
     const uint32_t tmem_base = *(volatile uint32_t*)&tp->tmem_base;
-    const unsigned int n_tiles = (unsigned int)((m + kSuperRows - 1) / kSuperRows);
+    const unsigned int n_tiles = (unsigned int)((m + kHalfRows - 1) / kHalfRows);
 
     if (warp == 0) {
-        if (!mlp_produce<GATHER>(tp, ring, &map_x, &map_w, p.g, n_tiles, p.row_idx, m, p.n_stored) && lane == 0) step_give_up(p, tp);
+        if (!mlp_produce<GATHER, kHalfRows, kHalfStages>(tp, ring, &map_x, &map_w, p.g, n_tiles, p.row_idx, m, p.n_stored) && lane == 0) step_give_up(p, tp);
     } else if (GATHER && (warp == 3 || warp >= 12)) {
-        if (!mlp_produce<GATHER>(tp, ring, &map_x, &map_w, p.g, n_tiles, p.row_idx, m, p.n_stored, warp == 3 ? 1 : warp - 10) && lane == 0)
+        if (!mlp_produce<GATHER, kHalfRows, kHalfStages>(tp, ring, &map_x, &map_w, p.g, n_tiles, p.row_idx, m, p.n_stored, warp == 3 ? 1 : warp - 10) && lane == 0)
             step_give_up(p, tp);
     } else if (warp == 1) {
-        if (!mlp_issue_mma(tp, ring, p.g, n_tiles, tmem_base) && lane == 0) step_give_up(p, tp);
+        if (!mlp_issue_mma<kHalfRows, kHalfStages>(tp, ring, p.g, n_tiles, tmem_base) && lane == 0) step_give_up(p, tp);
     } else if (warp >= 4 && warp < 12) {
         // ------------------------------------------------------------ epilogue
+        // warps 4..7 take this CTA's even tiles (accumulator 0), warps 8..11 the odd ones (accumulator 1)
         const int ew = warp - 4;
         const int quad = warp & 3, acc = ew >> 2;
-        const int row = acc * 128 + quad * 32 + lane;
+        const int row = quad * 32 + lane;
         const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kMaxHidden);
         const float bias2 = *p.b2;
         float sum_rh[kMaxHidden / 32], sum_p[kMaxHidden / 32];   // lane l: columns c0 + l of this warp's rows
 #pragma unroll
         for (int c = 0; c < kMaxHidden / 32; ++c) sum_rh[c] = sum_p[c] = 0.0f;
         float sum_r = 0.0f;
-        int it = 0;
-        for (unsigned int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
-            if (!mbar_wait(&tp->acc_full, (uint32_t)(it & 1), abort_flag)) {
+        int it = acc;
+        for (unsigned long long tile = blockIdx.x + (unsigned long long)acc * gridDim.x; tile < n_tiles; tile += 2ull * gridDim.x, it += 2) {
+            if (!mbar_wait(&tp->acc_full[acc], (uint32_t)((it >> 1) & 1), abort_flag)) {
                 if (lane == 0) step_give_up(p, tp);
                 break;
             }
             tc_fence_after_sync();
-            const int64_t i = (int64_t)tile * kSuperRows + row;
+            const int64_t i = (int64_t)tile * kHalfRows + row;
             // this row's loss and validity are requested before the pass over TMEM
             bool valid = i < m;
             float f_i = 0.0f;
@@ -214,7 +217,7 @@ mlp_residual_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
             }
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&tp->acc_empty);
+            if (lane == 0) mbar_arrive(&tp->acc_empty[acc]);
         }
 #pragma unroll
         for (int c = 0; c < kMaxHidden / 32; ++c) {
@@ -544,7 +547,7 @@ aa_status launch_assistant_step_mlp(aa_ctx_impl* c, const MlpFeat& f, float* W1_
     p.w2 = const_cast<float*>(f.w2);
     p.b2 = const_cast<float*>(f.b2);
     p.d = f.d;
-    p.g = make_mlp_geom(f.d, f.hidden);
+    p.g = make_mlp_geom(f.d, f.hidden, kHalfRows);
     p.Pt = static_cast<__nv_bfloat16*>(c->mlp_pt);
     p.pitch = (m_host + kSuperRows - 1) / kSuperRows * kSuperRows;
     p.small = c->mlp_small;
@@ -564,7 +567,7 @@ aa_status launch_assistant_step_mlp(aa_ctx_impl* c, const MlpFeat& f, float* W1_
     p.splits = (int)splits;
 
     alignas(64) CUtensorMap map_x, map_w, map_pt, map_xg;
-    if (!encode_bf16_tile_map(&map_x, f.x, (uint64_t)f.n, (uint64_t)f.d, (uint64_t)f.row_stride, gather ? 1 : kSuperRows) ||
+    if (!encode_bf16_tile_map(&map_x, f.x, (uint64_t)f.n, (uint64_t)f.d, (uint64_t)f.row_stride, gather ? 1 : kHalfRows) ||
         !encode_bf16_tile_map(&map_w, f.W1_bf16, (uint64_t)f.hidden, (uint64_t)f.d, (uint64_t)f.d, (uint32_t)f.hidden) ||
         !encode_bf16_tile_map(&map_pt, p.Pt, (uint64_t)f.hidden, (uint64_t)p.pitch, (uint64_t)p.pitch, (uint32_t)f.hidden) ||
         !encode_bf16_tile_map(&map_xg, f.x, (uint64_t)f.n, (uint64_t)f.d, (uint64_t)f.row_stride, gather ? 1 : kRowSlice))
@@ -572,11 +575,11 @@ aa_status launch_assistant_step_mlp(aa_ctx_impl* c, const MlpFeat& f, float* W1_
 
     // 1. forward + residuals + P^T
     {
-        const size_t smem = 1024 + (size_t)kMlpStages * p.g.stage_bytes + sizeof(float) * (2 * kMaxHidden + kStepEpiWarps * 2 * kMaxHidden) +
+        const size_t smem = 1024 + (size_t)kHalfStages * p.g.stage_bytes + sizeof(float) * (2 * kMaxHidden + kStepEpiWarps * 2 * kMaxHidden) +
                             sizeof(double) * (kStepMlpThreads / 32) + sizeof(float) * kStepEpiWarps + sizeof(TilePipe) + 64;
         const void* kernel = gather ? (const void*)mlp_residual_kernel<true> : (const void*)mlp_residual_kernel<false>;
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return AA_ERR_CUDA;
-        const int64_t tiles = (m_host + kSuperRows - 1) / kSuperRows;
+        const int64_t tiles = (m_host + kHalfRows - 1) / kHalfRows;
         int grid = max_ctas;
         if (grid > tiles) grid = (int)tiles;
         void* args[] = {&map_x, &map_w, &p};
