@@ -455,7 +455,8 @@ aa_status aa_device_status(aa_ctx* ctx, int32_t* latched) {
         // a scan that gave up may have left the ticket state half-used: re-arm everything
         const unsigned int zeros[4] = {0, 0, 0, 0};
         if (cudaMemcpyAsync(c->ctl, zeros, 2 * sizeof(unsigned int), cudaMemcpyHostToDevice, c->stream) != cudaSuccess ||
-            cudaMemsetAsync(&c->ctl->status, 0, sizeof(int) + 2 * sizeof(unsigned int), c->stream) != cudaSuccess ||   // status, sums_in, applied
+            cudaMemsetAsync(&c->ctl->status, 0, sizeof(int), c->stream) != cudaSuccess ||
+            cudaMemsetAsync(&c->ctl->sums_in, 0, 3 * sizeof(unsigned int), c->stream) != cudaSuccess ||   // sums_in, grad_done, applied
             cudaStreamSynchronize(c->stream) != cudaSuccess)
             return AA_ERR_CUDA;
     }

@@ -15,9 +15,13 @@ struct Control {
     unsigned int done;     // CTAs of the running scan kernel that have finished
     unsigned int epoch;    // generation of the look-back flags; bumped by the last CTA of each scan
     int status;            // first device-side condition latched (aa_status), 0 = none
+    unsigned int pad0[28];
+    // second 128-byte line: the counters the gradient kernel's CTAs poll, kept away from the ticket counter that the
+    // same kernel's producers hammer with atomics
     unsigned int sums_in;  // CTAs of the running gradient kernel that have published their share of the loss sum
+    unsigned int grad_done;  // CTAs of the running gradient kernel that have written their partial sums
     unsigned int applied;  // CTAs of the running gradient kernel that have seen every CTA's partial sums
-    unsigned int pad[58];
+    unsigned int pad1[29];
 };
 static_assert(sizeof(Control) == 256, "control block is one 256-byte line group");
 

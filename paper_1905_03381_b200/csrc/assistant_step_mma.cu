@@ -60,6 +60,7 @@ struct MmaControl {
     float part[kMStages][kMWarps][kFragRows];     // each warp's share of the dot products
     alignas(4) __nv_bfloat16 r_split[kMWarps][3][kFragRows];   // per warp: hi / mid / lo terms of the residuals
     double red[kMWarps];
+    double T_mean;
     float bias_sum;
     int stop_j;
     int abort_flag;
@@ -129,16 +130,16 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_mma_kernel(StepParam
             if (tk >= n_tickets || i >= m) return -1;
             return g.contiguous ? (long long)i : batch_row(p, i);
         };
-        unsigned int cur = 0, next = 0;
-        if (lane == 0) cur = atomicAdd(&p.ctl->ticket, 1u);
-        cur = __shfl_sync(0xFFFFFFFFu, cur, 0);
+        // the first ticket of a CTA is its block index (no round trip before the first copies); the counter hands
+        // out the tickets from gridDim.x on
+        unsigned int cur = blockIdx.x, next = 0;
         long long cur_row = fetch_row(cur);
-        if (lane == 0) next = atomicAdd(&p.ctl->ticket, 1u);
+        if (lane == 0) next = gridDim.x + atomicAdd(&p.ctl->ticket, 1u);
         while (ok && cur < n_tickets) {
             next = __shfl_sync(0xFFFFFFFFu, next, 0);
             const long long next_row = fetch_row(next);       // on its way while this ticket is issued
             unsigned int after = 0;
-            if (lane == 0) after = atomicAdd(&p.ctl->ticket, 1u);
+            if (lane == 0) after = gridDim.x + atomicAdd(&p.ctl->ticket, 1u);
             for (int s = 0; s < kMTicketRows / kMRows; ++s) {
                 const int64_t i0 = (int64_t)cur * kMTicketRows + (int64_t)s * kMRows;
                 if (i0 >= m) break;
@@ -188,6 +189,11 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_mma_kernel(StepParam
         const int cw = warp - 1;
         const int ct = tid - 32;
         // weights as three bf16 planes, and the batch-mean threshold (fixed order: thread stride, warp tree, warp index)
+        const bool mean_T = p.thresh_mode != AA_THRESH_VALUE;
+        // this CTA's slice of the losses (batch-mean threshold): the first load is issued ahead of the weight loads
+        const int64_t per = ((m + gridDim.x - 1) / gridDim.x + 3) / 4 * 4;
+        const int64_t s_lo = (int64_t)blockIdx.x * per, s_hi = s_lo + per < m ? s_lo + per : m;
+        const float first_loss = (mean_T && s_lo + ct < s_hi) ? __ldg(p.loss + s_lo + ct) : 0.0f;
         for (int jf = ct; jf < g.d; jf += kMWarps * 32) {
             __nv_bfloat16 hi, mid, lo;
             split3(__ldcg(p.f.w + jf), hi, mid, lo);       // w is rewritten at the end of this kernel: no read-only path
@@ -199,12 +205,9 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_mma_kernel(StepParam
         // one slice (fixed order: thread stride, warp tree, warp index), publishes its share, and all CTAs add the shares
         // in one fixed order once everyone has published (by then the first dot products are done).
         double T_shrink = (double)p.threshold;
-        const bool mean_T = p.thresh_mode != AA_THRESH_VALUE;
         if (mean_T) {
-            const int64_t per = ((m + gridDim.x - 1) / gridDim.x + 3) / 4 * 4;
-            const int64_t lo = (int64_t)blockIdx.x * per, hi = lo + per < m ? lo + per : m;
-            double acc = 0.0;
-            for (int64_t i = lo + ct; i < hi; i += kMWarps * 32) acc += (double)__ldg(p.loss + i);
+            double acc = (double)first_loss;
+            for (int64_t i = s_lo + ct + kMWarps * 32; i < s_hi; i += kMWarps * 32) acc += (double)__ldg(p.loss + i);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
             if (lane == 0) cb->red[cw] = acc;
@@ -279,22 +282,33 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_mma_kernel(StepParam
                 break;
             }
             if (!have_T) {
-                // every CTA's share of the loss sum, added in CTA order (identical in every warp of every CTA)
-                unsigned int polls = 0;
-                while (*(volatile unsigned int*)&p.ctl->sums_in < gridDim.x && !*abort_flag) {
-                    if (++polls > kSpinLimit) break;
-                    __nanosleep(40);
-                }
-                if (*(volatile unsigned int*)&p.ctl->sums_in < gridDim.x) {
-                    if (lane == 0) mma_give_up(p, cb);
-                    break;
-                }
-                __threadfence();
-                double total = 0.0;   // lane l adds shares l, l + 32, ...; then a fixed shuffle tree: the same order everywhere
-                for (unsigned int q = lane; q < gridDim.x; q += 32) total += __ldcg(p.loss_sums + q);
+                // every CTA's share of the loss sum, added in CTA order (the same order in every CTA).  One warp polls
+                // and adds; the others meet it at a named barrier.
+                if (cw == 0) {
+                    unsigned int polls = 0;
+                    while (*(volatile unsigned int*)&p.ctl->sums_in < gridDim.x && !*abort_flag) {
+                        if (++polls > kSpinLimit) break;
+                        __nanosleep(32);
+                    }
+                    if (*(volatile unsigned int*)&p.ctl->sums_in < gridDim.x) {
+                        if (lane == 0) mma_give_up(p, cb);
+                    } else {
+                        __threadfence();
+                        double share[5];      // lane l adds shares l, l + 32, ... (loads in flight together); then a fixed shuffle tree
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xFFFFFFFFu, total, o);
-                T_shrink = m > 0 ? total / (double)m : 0.0;
+                        for (int u = 0; u < 5; ++u) share[u] = lane + 32u * u < gridDim.x ? __ldcg(p.loss_sums + lane + 32 * u) : 0.0;
+                        double total = 0.0;
+#pragma unroll
+                        for (int u = 0; u < 5; ++u) total += share[u];
+                        for (unsigned int q = lane + 160; q < gridDim.x; q += 32) total += __ldcg(p.loss_sums + q);
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xFFFFFFFFu, total, o);
+                        if (lane == 0) cb->T_mean = m > 0 ? total / (double)m : 0.0;
+                    }
+                }
+                asm volatile("bar.sync 3, %0;" ::"n"(kMWarps * 32) : "memory");
+                if (*abort_flag) break;
+                T_shrink = cb->T_mean;
                 have_T = true;
             }
             // ---- residuals of the 16 rows (every warp, lanes 0..15), split into three bf16 terms
@@ -359,6 +373,12 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_mma_kernel(StepParam
             if (lane == 0) cb->bias_sum = bias_acc;
         }
     }
+    // the weights this CTA will update are read while the partial sums of the other CTAs are still on their way
+    const int cols_per_cta = (g.d + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int c0 = (int)blockIdx.x * cols_per_cta;
+    const int c1 = c0 + cols_per_cta < g.d ? c0 + cols_per_cta : g.d;
+    float w_first = 0.0f;
+    if (warp == 0 && c0 + lane < c1) w_first = __ldcg(p.w + c0 + lane);
     __syncthreads();
     // ---------------------------------------------------------------- update (Algorithm 2: Assistant.update)
     // Every CTA publishes its sums, waits (bounded) until all CTAs of this cooperative launch have done so, then adds
@@ -366,13 +386,13 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_mma_kernel(StepParam
     if (tid == 0) {
         p.partials[(int64_t)gridDim.x * p.d_pad + blockIdx.x] = cb->bias_sum;
         __threadfence();
-        atomicAdd(&p.ctl->done, 1u);
+        atomicAdd(&p.ctl->grad_done, 1u);
         unsigned int polls = 0;
-        while (*(volatile unsigned int*)&p.ctl->done < gridDim.x && !*abort_flag) {
+        while (*(volatile unsigned int*)&p.ctl->grad_done < gridDim.x && !*abort_flag) {
             if (++polls > kSpinLimit) break;
             __nanosleep(64);
         }
-        if (*(volatile unsigned int*)&p.ctl->done < gridDim.x || *abort_flag) {
+        if (*(volatile unsigned int*)&p.ctl->grad_done < gridDim.x || *abort_flag) {
             mma_give_up(p, cb);
         } else {
             __threadfence();
@@ -380,7 +400,7 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_mma_kernel(StepParam
             const unsigned int prev = atomicAdd(&p.ctl->applied, 1u);
             if (prev == gridDim.x - 1) {
                 p.ctl->ticket = 0;
-                p.ctl->done = 0;
+                p.ctl->grad_done = 0;
                 p.ctl->sums_in = 0;
                 p.ctl->applied = 0;
             }
@@ -391,16 +411,20 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_mma_kernel(StepParam
     {
         float* share = reinterpret_cast<float*>(x_ring);            // [warps][32]; every copy into the ring has landed
         constexpr int kAllWarps = kMThreads / 32;
-        const int cols_per_cta = (g.d + (int)gridDim.x - 1) / (int)gridDim.x;
-        const int c0 = (int)blockIdx.x * cols_per_cta;
-        const int c1 = c0 + cols_per_cta < g.d ? c0 + cols_per_cta : g.d;
         const float scale = p.lr / (float)m;
         for (int cb0 = c0; cb0 < c1; cb0 += 32) {
             const int jcol = cb0 + lane;
             float gsum = 0.0f;
             if (jcol < c1) {
-#pragma unroll 4
-                for (unsigned int q = warp; q < gridDim.x; q += kAllWarps) gsum += __ldcg(p.partials + (int64_t)q * p.d_pad + jcol);
+                float part_v[12];   // 148 CTAs over 13 warps: at most 12 partials per lane, all loads in flight together
+#pragma unroll
+                for (int u = 0; u < 12; ++u) {
+                    const unsigned int q = warp + u * kAllWarps;
+                    part_v[u] = q < gridDim.x ? __ldcg(p.partials + (int64_t)q * p.d_pad + jcol) : 0.0f;
+                }
+#pragma unroll
+                for (int u = 0; u < 12; ++u) gsum += part_v[u];
+                for (unsigned int q = warp + 12 * kAllWarps; q < gridDim.x; q += kAllWarps) gsum += __ldcg(p.partials + (int64_t)q * p.d_pad + jcol);
             }
             share[warp * 32 + lane] = gsum;
             __syncthreads();
@@ -408,7 +432,7 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_mma_kernel(StepParam
                 float t = 0.0f;
 #pragma unroll
                 for (int k = 0; k < kAllWarps; ++k) t += share[k * 32 + lane];
-                const float w_old = __ldcg(p.w + jcol);
+                const float w_old = cb0 == c0 ? w_first : __ldcg(p.w + jcol);
                 p.w[jcol] = p.adam.on ? adam_update(p.adam, w_old, t / (float)m, p.lr, jcol) : w_old - scale * t;
             }
             __syncthreads();
