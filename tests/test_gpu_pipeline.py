@@ -120,3 +120,67 @@ def test_depth_changes_batches_and_reruns_agree(data):
         assert len(s1 ^ s2) <= 2
     # batches 0..2 were screened before the first update in both runs of depth 2, batch 0 in every run
     assert np.array_equal(a["idx"][0][: int(a["count"][0])], b1["idx"][0][: int(b1["count"][0])])
+
+
+def test_pipeline_with_csr_features_and_adam():
+    """The same schedule over bag-of-words pools with the Adam update: every batch against the oracle's screening with
+    the GPU's parameter snapshot of its lag, every update against the oracle's gradient and Adam rule from the GPU's
+    own state before it (parameters and moments: |p - p_ref| <= 2e-4 |p_ref| + 2e-4 rms(p_ref))."""
+    build.build()
+    n, d, steps, depth = 3000, 1 << 12, 4, 1
+    lr, b1, b2, eps = 0.01, 0.9, 0.999, 1e-5
+    rng = np.random.default_rng(5)
+    pools = []
+    for j in range(steps):
+        lens = rng.integers(1, 50, n)
+        indptr = np.zeros(n + 1, np.int32); indptr[1:] = np.cumsum(lens)
+        col = rng.integers(0, d, int(indptr[-1])).astype(np.int32)
+        val = rng.integers(1, 4, int(indptr[-1])).astype(np.float32)
+        pools.append((indptr, col, val) + tuple(torch.from_numpy(a).to(DEV) for a in (indptr, col, val)))
+    logits = [W.normal((n, 20), 2.0, 800 + j, torch.float32, DEV) for j in range(steps)]
+    labels = [W.randint(0, 20, (n,), 900 + j, DEV).to(torch.int32) for j in range(steps)]
+    w = W.normal((d,), 0.3, 11, torch.float32, DEV)
+    b = torch.full((1,), -0.2, dtype=torch.float32, device=DEV)
+    w0, b0 = w.cpu().numpy().copy(), np.float32(-0.2)
+    mom, var = torch.zeros(d + 1, device=DEV), torch.zeros(d + 1, device=DEV)
+    state = B.adam_state(mom, var, b1, b2, eps)
+    hist = {k: torch.zeros((steps, d + 1), device=DEV) for k in ("p", "m", "v")}
+    pipe = StreamPipeline(depth, max_rows=n, max_d=d, capacity=n, device=DEV, slots=steps)
+
+    def features(j, row_idx):
+        return B.csr_features(pools[j][3], pools[j][4], pools[j][5], d, row_idx=row_idx)
+
+    def boss(t, ctx, idx, count_dev, out_loss):
+        ctx.aa_instance_loss(B.logits_desc(logits[t]), labels[t], out_loss, count_dev=count_dev)
+
+    def after_update(t):
+        hist["p"][t, :d].copy_(w); hist["p"][t, d:].copy_(b)
+        hist["m"][t].copy_(mom); hist["v"][t].copy_(var)
+
+    pipe.run(steps, features, boss, B.linear_assistant(w, b), 0.2, 9, lr, adam=state, after_update=after_update)
+    torch.cuda.synchronize()
+    assert pipe.device_status() == B.AA_OK and state.t == steps
+    idx, cnt, loss = pipe.idx.cpu().numpy(), pipe.count.cpu().numpy()[:, 0], pipe.loss.cpu().numpy()
+    P, M, V = (hist[k].cpu().numpy() for k in ("p", "m", "v"))
+    pipe.close()
+    snaps = [np.concatenate([w0, [b0]])] + [P[t] for t in range(steps)]
+    moms = [(np.zeros(d + 1, np.float32), np.zeros(d + 1, np.float32))] + [(M[t], V[t]) for t in range(steps)]
+    ids = np.arange(n)
+    for j in range(steps):
+        ph = snaps[max(0, j - depth)]
+        s = O.score_csr(pools[j][0], pools[j][1], pools[j][2], ph[:d], ph[d])
+        g = O.sigmoid(s)
+        keep, p_acc, c = O.shrink(g, 0.2, 9, j), O.accept_prob(g, 0.2), O.uniform(9, j, ids)
+        got = np.zeros(n, np.uint8); got[idx[j][: cnt[j]]] = 1
+        assert np.all(np.abs(p_acc - c)[got != keep] < 1e-5), f"batch {j}"
+    for t in range(steps):
+        m_t = int(cnt[t]); Bt = idx[t][:m_t].astype(np.int32); f = loss[t][:m_t]
+        assert np.all(np.abs(f - O.row_loss(logits[t].cpu().numpy()[:m_t], labels[t].cpu().numpy()[:m_t])) <= 1e-4)
+        z = O.labels(f, O.batch_mean(f))
+        s = O.score_csr(pools[t][0], pools[t][1], pools[t][2], snaps[t][:d], snaps[t][d], row_idx=Bt, n_cand=m_t)
+        gw, gb = O.linear_grad_csr(pools[t][0], pools[t][1], pools[t][2], d, s, z, row_idx=Bt)
+        p_ref, m_ref, v_ref = O.adam(snaps[t], moms[t][0], moms[t][1], np.concatenate([gw, [gb]]), lr, b1, b2, eps, t + 1)
+        for got_a, ref_a in ((P[t], p_ref), (M[t], m_ref), (V[t], v_ref)):
+            ref64 = ref_a.astype(np.float64)
+            tol = 2e-4 * np.abs(ref64) + 2e-4 * np.sqrt(np.mean(ref64 ** 2) + 1e-300)
+            assert np.all(np.abs(got_a - ref64) <= tol)
