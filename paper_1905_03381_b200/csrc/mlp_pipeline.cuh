@@ -3,7 +3,8 @@
 // for one super-tile of 256 rows at a time, two 128-row fp32 accumulators side by side in TMEM.
 //
 //   producer warp : per 64-wide K-slice, 256 feature rows x 64 columns and `hidden` W1 rows x 64
-//                   columns (128-byte swizzle) into a 3-stage ring.  Rows come as one TMA box
+//                   columns (128-byte swizzle) into a 3-stage ring (the gradient's forward pass: 128
+//                   rows per tile, 4 stages, the two accumulators alternating between tiles).  Rows come as one TMA box
 //                   when the tile's rows are adjacent in memory, or as 64 four-row gathers
 //                   (tile::gather4, spread over eight warps) when a row list selects them.
 //   MMA warp      : tcgen05.mma M = 128, N = hidden, K = 16, eight per stage; commits every
@@ -84,7 +85,7 @@ template <bool GATHER, int ROWS = kSuperRows, int STAGES = kMlpStages>
 __device__ __forceinline__ bool mlp_produce(TilePipe* tp, unsigned char* ring, const CUtensorMap* map_x, const CUtensorMap* map_w,
                                             const MlpGeom& g, unsigned int n_tiles, const int32_t* rows, long long n_list,
                                             long long n_stored, int part = 0) {
-    // Gathered rows are fetched by kGatherWarps warps (part = 0 .. kGatherWarps - 1), 32 rows each, one four-row
+    // Gathered rows are fetched by kGatherWarps warps (part = 0 .. kGatherWarps - 1), ROWS / kGatherWarps rows each, one four-row
     // gather per issuing lane and stage: the gathers a single warp issues retire at only about one per 43 ns.  Part 0 is the
     // producer proper (it also posts the expected bytes and loads W1); the others follow the same barriers.
     const int lane = threadIdx.x & 31;

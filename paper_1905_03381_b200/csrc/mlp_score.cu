@@ -4,11 +4,12 @@
 // tcgen05 tensor cores (Sec. 5.2 asks only for a light-weight classifier g; this is the
 // library's dense-contraction Assistant).
 //
-// One persistent CTA per SM, 12 warps.  A CTA owns super-tiles of 256 candidates: two 128-row
+// One persistent CTA per SM, 12 warps (18 when a candidate list selects the rows: warps 3 and 12..17
+// then issue row gathers beside warp 0).  A CTA owns super-tiles of 256 candidates: two 128-row
 // accumulators [128 x hidden] fp32 side by side in tensor memory, so that every 64-wide K-slice
 // of W1 fetched into shared memory is used for 256 candidates.
 //   warp 0      : TMA producer.  Per K-slice 256 feature rows x 64 columns (one box, or 64
-//                 four-row gathers when a candidate list selects the rows) and one box of
+//                 four-row gathers spread over eight warps when a candidate list selects the rows) and one box of
 //                 `hidden` W1 rows x 64 columns (128-byte swizzle) into a 3-stage ring.
 //   warp 1      : issues tcgen05.mma (M = 128, N = hidden, K = 16; 8 per stage), commits each
 //                 stage back to the producer and the finished super-tile to the epilogue.
