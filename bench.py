@@ -212,7 +212,7 @@ def workload_config(cfg, args, reference=False):
         "pool_rows": cfg.n, "d": cfg.d, "classes": cfg.classes, "mix": cfg.gamma, "lr": cfg.lr,
         "pools_rotated": None if reference else args.pools,
         "l2_policy": "inputs larger than L2: each pool is 403 MB and pools rotate",
-        "stage_events": f"per-stage CUDA events on every {EVENT_EVERY}th timed step",
+        "stage_events": None if reference else f"per-stage CUDA events on every {EVENT_EVERY}th timed step",
         "parallelism": f"instance-sharded x{args.gpus}, one Assistant per GPU, no data-path collective",
     }
 
