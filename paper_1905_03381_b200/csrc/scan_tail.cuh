@@ -57,10 +57,11 @@ __device__ __forceinline__ int lookback_exclusive(const ShrinkParams& p, unsigne
         return 0;
     }
     if (lane == 0) st_relaxed_u64(&state[tile], pack_state(flag_agg, total));
-    // Each poll reads kLookWide*32 predecessor states in one round trip (lane l, group j ->
-    // tile window_end - j*32 - l): when every SM runs in step, the nearest finished prefix is
-    // about one tile per SM back, and a 32-wide window would need a chain of dependent reads.
-    constexpr int kLookWide = 8;
+    // Each poll reads the 32 predecessor states just before the window's end (lane l -> tile window_end - l) and the
+    // window moves back by the groups that were complete.  Wider polls (256 states per round trip, to reach the
+    // nearest finished prefix in one step when every SM runs in step) were measured: the extra loads of ~600 polling
+    // warps cost the streaming kernels 7-9 % of their bandwidth and the scan-only kernels 10-20 % of their time.
+    constexpr int kLookWide = 1;
     int excl = 0;          // committed sum of fully scanned groups (same in every lane)
     long long window_end = (long long)tile - 1;
     bool gave_up = false, found = false;
