@@ -69,6 +69,72 @@ __global__ void __launch_bounds__(256) row_loss_group_kernel(LossParams p) {
     }
 }
 
+// Very short aligned rows (at most kShortVecs 16-byte vectors per lane): the whole row sits in registers, so the row
+// maximum is taken first and the sum second (no running rescale), and the loads of a row - label, every vector, and the
+// device row count - are all issued before anything is consumed: one memory round trip, then the label's logit from L1.
+constexpr int kShortVecs = 4;
+template <typename T, int LPR>
+__global__ void __launch_bounds__(256) row_loss_short_kernel(LossParams p) {
+    constexpr int VE = Vec<T>::kElems;
+    const int64_t rows_host = p.rows;
+    int64_t rows = rows_host;
+    int32_t count_raw = 0;
+    if (p.count_dev) count_raw = __ldg(p.count_dev);
+    const int gl = threadIdx.x % LPR;
+    const int nvec = (int)(p.cols / VE);
+    const int64_t groups_per_grid = (int64_t)gridDim.x * (blockDim.x / LPR);
+    const int64_t group0 = (int64_t)blockIdx.x * (blockDim.x / LPR) + threadIdx.x / LPR;
+    const int64_t rounds = (rows_host + groups_per_grid - 1) / groups_per_grid;
+    const T* base = static_cast<const T*>(p.logits);
+    for (int64_t it = 0; it < rounds; ++it) {
+        const int64_t r = group0 + it * groups_per_grid;
+        const bool inb = r < rows_host;
+        const T* row = base + (inb ? r : 0) * p.row_stride;
+        int y = inb ? __ldg(p.labels + r) : -1;
+        float x[kShortVecs][VE];
+#pragma unroll
+        for (int q = 0; q < kShortVecs; ++q) {
+            const int v = gl + q * LPR;
+            if (inb && v < nvec) {
+                Vec<T>::load(row + (int64_t)v * VE, x[q]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < VE; ++e) x[q][e] = -INFINITY;
+            }
+        }
+        if (p.count_dev) rows = count_raw < 0 ? 0 : ((int64_t)count_raw < rows_host ? (int64_t)count_raw : rows_host);
+        const bool live = r < rows;
+        if (live && y >= p.cols) {
+            latch(p.ctl, AA_ERR_BAD_INDEX);
+            y = -1;
+        }
+        const float label_logit = (live && y >= 0) ? Vec<T>::one(row + y) : 0.0f;
+        float m = -INFINITY;
+#pragma unroll
+        for (int q = 0; q < kShortVecs; ++q)
+#pragma unroll
+            for (int e = 0; e < VE; ++e) m = fmaxf(m, x[q][e]);
+#pragma unroll
+        for (int o = LPR / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+        const float neg_ref = m == -INFINITY ? 0.0f : -m * kLog2e;
+        float s0 = 0.0f, s1 = 0.0f;
+#pragma unroll
+        for (int q = 0; q < kShortVecs; ++q)
+#pragma unroll
+            for (int e = 0; e < VE; e += 2) {
+                s0 += ex2_approx(fmaf(x[q][e], kLog2e, neg_ref));
+                s1 += ex2_approx(fmaf(x[q][e + 1], kLog2e, neg_ref));
+            }
+        float ssum = s0 + s1;
+#pragma unroll
+        for (int o = LPR / 2; o > 0; o >>= 1) ssum += __shfl_xor_sync(0xFFFFFFFFu, ssum, o);
+        if (gl == 0 && live) {
+            RunState st = {m * kLog2e, ssum};
+            p.out[r] = y >= 0 ? finish_row(st, label_logit) : 0.0f;
+        }
+    }
+}
+
 // Long rows: one CTA per row.
 template <typename T>
 __global__ void __launch_bounds__(kRowThreads) row_loss_cta_kernel(LossParams p) {
@@ -135,6 +201,17 @@ aa_status launch_rows(aa_ctx_impl* c, LossParams& p) {
         int lpr = 2;
         while (lpr < 32 && lpr * 4 <= work) lpr <<= 1;   // two to four vectors per lane
         threads = 256;
+        const bool short_rows = !p.row_idx && row_bytes % 16 == 0 && (uintptr_t)p.logits % 16 == 0 && (p.row_stride * es) % 16 == 0 &&
+                                work <= (int64_t)lpr * kShortVecs;
+        if (short_rows) {
+            switch (lpr) {
+                case 2: kernel = (const void*)row_loss_short_kernel<T, 2>; break;
+                case 4: kernel = (const void*)row_loss_short_kernel<T, 4>; break;
+                case 8: kernel = (const void*)row_loss_short_kernel<T, 8>; break;
+                case 16: kernel = (const void*)row_loss_short_kernel<T, 16>; break;
+                default: kernel = (const void*)row_loss_short_kernel<T, 32>; lpr = 32; break;
+            }
+        } else
         switch (lpr) {
             case 2: kernel = (const void*)row_loss_group_kernel<T, 2>; break;
             case 4: kernel = (const void*)row_loss_group_kernel<T, 4>; break;
