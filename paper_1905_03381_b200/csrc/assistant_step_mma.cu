@@ -53,6 +53,7 @@ struct MmaGeometry {
 
 struct MmaControl {
     uint64_t x_full[kMStages], x_empty[kMStages], dots_in[kMStages];
+    uint64_t t_ready;                         // the batch-mean threshold is in T_mean (posted by the producer warp)
     long long first_row[kMStages];
     unsigned int valid[kMStages];
     alignas(16) float loss[kMStages][kMRows];
@@ -108,6 +109,7 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_mma_kernel(StepParam
             mbar_init(&cb->x_empty[s], kMWarps);
             mbar_init(&cb->dots_in[s], kMWarps);
         }
+        mbar_init(&cb->t_ready, 1);
         cb->bias_sum = 0.0f;
         cb->stop_j = 0x7FFFFFFF;
         cb->abort_flag = 0;
@@ -132,6 +134,35 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_mma_kernel(StepParam
         };
         // the first ticket of a CTA is its block index (no round trip before the first copies); the counter hands
         // out the tickets from gridDim.x on
+        // The batch-mean threshold: once the ring is full (or the batch has run out) this warp, idle until a stage is
+        // released, waits for every CTA's share of the loss sum, adds them in CTA order and posts the mean.
+        bool t_posted = p.thresh_mode == AA_THRESH_VALUE;
+        auto post_threshold = [&]() {
+            unsigned int polls = 0;
+            while (*(volatile unsigned int*)&p.ctl->sums_in < gridDim.x && !*abort_flag) {
+                if (++polls > kSpinLimit) break;
+                __nanosleep(32);
+            }
+            if (*(volatile unsigned int*)&p.ctl->sums_in < gridDim.x) {
+                if (lane == 0) mma_give_up(p, cb);
+            } else {
+                __threadfence();
+                double share[5];      // lane l adds shares l, l + 32, ... (loads in flight together); then a fixed shuffle tree
+#pragma unroll
+                for (int u = 0; u < 5; ++u) share[u] = lane + 32u * u < gridDim.x ? __ldcg(p.loss_sums + lane + 32 * u) : 0.0;
+                double total = 0.0;
+#pragma unroll
+                for (int u = 0; u < 5; ++u) total += share[u];
+                for (unsigned int q = lane + 160; q < gridDim.x; q += 32) total += __ldcg(p.loss_sums + q);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xFFFFFFFFu, total, o);
+                if (lane == 0) {
+                    cb->T_mean = m > 0 ? total / (double)m : 0.0;
+                    mbar_arrive(&cb->t_ready);
+                }
+            }
+            t_posted = true;
+        };
         unsigned int cur = blockIdx.x, next = 0;
         long long cur_row = fetch_row(cur);
         if (lane == 0) next = gridDim.x + atomicAdd(&p.ctl->ticket, 1u);
@@ -143,6 +174,7 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_mma_kernel(StepParam
             for (int s = 0; s < kMTicketRows / kMRows; ++s) {
                 const int64_t i0 = (int64_t)cur * kMTicketRows + (int64_t)s * kMRows;
                 if (i0 >= m) break;
+                if (j >= kMStages && !t_posted) post_threshold();
                 if (j >= kMStages && !mbar_wait(&cb->x_empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
                 unsigned char* dst = x_ring + (size_t)stage * g.stage_bytes;
                 const long long r = __shfl_sync(0xFFFFFFFFu, cur_row, (s * kMRows + lane) & 31);
@@ -168,6 +200,7 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_mma_kernel(StepParam
             cur_row = next_row;
             next = after;
         }
+        if (!t_posted) post_threshold();
         if (ok) {
             // one empty stage wakes the compute warps for the last time
             if (lane == 0) *(volatile int*)&cb->stop_j = j;
@@ -203,7 +236,7 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_mma_kernel(StepParam
         }
         // Batch-mean threshold: summing all M losses in every CTA costs more than the first ring stage, so each CTA adds
         // one slice (fixed order: thread stride, warp tree, warp index), publishes its share, and all CTAs add the shares
-        // in one fixed order once everyone has published (by then the first dot products are done).
+        // in one fixed order once everyone has published (the producer warp does that while the ring is full).
         double T_shrink = (double)p.threshold;
         if (mean_T) {
             double acc = (double)first_loss;
@@ -282,33 +315,12 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_mma_kernel(StepParam
                 break;
             }
             if (!have_T) {
-                // every CTA's share of the loss sum, added in CTA order (the same order in every CTA).  One warp polls
-                // and adds; the others meet it at a named barrier.
-                if (cw == 0) {
-                    unsigned int polls = 0;
-                    while (*(volatile unsigned int*)&p.ctl->sums_in < gridDim.x && !*abort_flag) {
-                        if (++polls > kSpinLimit) break;
-                        __nanosleep(32);
-                    }
-                    if (*(volatile unsigned int*)&p.ctl->sums_in < gridDim.x) {
-                        if (lane == 0) mma_give_up(p, cb);
-                    } else {
-                        __threadfence();
-                        double share[5];      // lane l adds shares l, l + 32, ... (loads in flight together); then a fixed shuffle tree
-#pragma unroll
-                        for (int u = 0; u < 5; ++u) share[u] = lane + 32u * u < gridDim.x ? __ldcg(p.loss_sums + lane + 32 * u) : 0.0;
-                        double total = 0.0;
-#pragma unroll
-                        for (int u = 0; u < 5; ++u) total += share[u];
-                        for (unsigned int q = lane + 160; q < gridDim.x; q += 32) total += __ldcg(p.loss_sums + q);
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xFFFFFFFFu, total, o);
-                        if (lane == 0) cb->T_mean = m > 0 ? total / (double)m : 0.0;
-                    }
+                // the producer warp posts the mean once every CTA's share is in
+                if (!mbar_wait(&cb->t_ready, 0, abort_flag)) {
+                    if (lane == 0) mma_give_up(p, cb);
+                    break;
                 }
-                asm volatile("bar.sync 3, %0;" ::"n"(kMWarps * 32) : "memory");
-                if (*abort_flag) break;
-                T_shrink = cb->T_mean;
+                T_shrink = *(volatile double*)&cb->T_mean;
                 have_T = true;
             }
             // ---- residuals of the 16 rows (every warp, lanes 0..15), split into three bf16 terms
