@@ -36,7 +36,6 @@ constexpr int kTmaThreads = (kConsumers + 1 + kTails) * 32;   // warp 0 producer
 constexpr int kSlotShift = 3;
 constexpr int kScoreSlots = 1 << kSlotShift;         // tiles in flight between consumers and tails
 constexpr int kMaxUnits = 8;                         // 32-candidate units per tile
-constexpr int kMaxTmaTileRows = kMaxUnits * 32;
 
 struct TmaGeometry {
     int chunk_rows;        // rows per ring stage (power of two <= 32)
