@@ -560,3 +560,34 @@ def test_instance_loss_rows_bad_entry_latches_and_gives_zero():
     assert got[1] == 0.0 and got[2] == 0.0 and got[0] > 0 and got[3] > 0
     assert ctx.aa_device_status() == B.AA_OK
     ctx.close()
+
+
+# --------------------------------------------------------------------------
+# short aligned rows (the register-resident loss kernel): widths at and around its limits, extreme logits
+# --------------------------------------------------------------------------
+
+@pytest.mark.parametrize("rows,cols,dtype", [
+    (5000, 4, torch.float32), (333, 8, torch.float32), (2049, 16, torch.float32), (4100, 100, torch.float32),
+    (1000, 128, torch.float32), (1000, 132, torch.float32), (777, 8, torch.bfloat16), (1025, 64, torch.bfloat16),
+    (3000, 256, torch.bfloat16), (500, 264, torch.bfloat16), (1, 32, torch.float32),
+])
+def test_short_row_losses(aa, rows, cols, dtype):
+    logits = W.normal((rows, cols), 3.0, rows + 3 * cols, dtype, DEV)
+    labels = W.randint(0, cols, (rows,), rows + cols, DEV)
+    if rows > 10:
+        labels[3] = -1                                    # padding row
+        logits[5] = 80.0 if dtype == torch.float32 else 64.0     # all equal and large: loss = ln(cols)
+        logits[7, :] = -1e30 if dtype == torch.float32 else -3e38  # one finite winner among hugely negative logits
+        logits[7, cols - 1] = 2.0
+        labels[7] = cols - 1
+    count = rows if rows < 10 else rows - 4                   # the device count cuts the last rows off
+    out = torch.full((rows,), -3.0, dtype=torch.float32, device=DEV)
+    cnt_t = torch.tensor([count], dtype=torch.int32, device=DEV)
+    aa.aa_instance_loss(B.logits_desc(logits), labels, out, count_dev=cnt_t)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy()
+    ref = O.row_loss(W.to_oracle(logits), labels.cpu().numpy())
+    assert np.max(np.abs(got[:count] - ref[:count])) <= 1e-4, float(np.max(np.abs(got[:count] - ref[:count])))
+    assert np.all(got[count:] == -3.0)
+    if rows > 10:
+        assert got[3] == 0.0 and abs(got[5] - math.log(cols)) <= 1e-4 and abs(got[7]) <= 1e-6
