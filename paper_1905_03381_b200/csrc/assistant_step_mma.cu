@@ -485,7 +485,13 @@ aa_status launch_assistant_grad_dense_mma(aa_ctx_impl* c, StepParams& p, int* pa
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return AA_ERR_CUDA;
     void* args[] = {&p, &g};
     // cooperative: the CTAs wait for one another before the update, so all of them must be resident at once
-    if (cudaLaunchCooperativeKernel(kernel, dim3(grid), dim3(kMThreads), args, smem, c->stream) != cudaSuccess) return AA_ERR_CUDA;
+    const cudaError_t le = cudaLaunchCooperativeKernel(kernel, dim3(grid), dim3(kMThreads), args, smem, c->stream);
+    if (le == cudaErrorCooperativeLaunchTooLarge || le == cudaErrorNotSupported) {
+        // the device cannot hold the whole grid at once (or has no cooperative launch): the other gradient kernels wait on nobody
+        (void)cudaGetLastError();
+        return AA_ERR_UNSUPPORTED;
+    }
+    if (le != cudaSuccess) return AA_ERR_CUDA;
     ++c->launches;
     *parts_out = 0;   // the update was taken inside the kernel
     return AA_OK;
