@@ -24,8 +24,21 @@ __device__ __forceinline__ void scan_row(RunState& st, const T* row, int64_t col
     const int64_t nvec = (cols - head) / VE;
     const int64_t tail0 = head + nvec * VE;
     const T* body = row + head;
-#pragma unroll 2
-    for (int64_t v = rank; v < nvec; v += nthreads) {
+    constexpr int K = 4;                    // vectors per trip that share the running-maximum bookkeeping
+    int64_t v = rank;
+    for (; v + (K - 1) * (int64_t)nthreads < nvec; v += K * (int64_t)nthreads) {
+        float x[K][VE];
+#pragma unroll
+        for (int k = 0; k < K; ++k) Vec<T>::load(body + (v + k * (int64_t)nthreads) * VE, x[k]);
+        absorb_vecs<K, VE>(st, x);
+    }
+    for (; v + (int64_t)nthreads < nvec; v += 2 * (int64_t)nthreads) {
+        float x[2][VE];
+        Vec<T>::load(body + v * VE, x[0]);
+        Vec<T>::load(body + (v + nthreads) * VE, x[1]);
+        absorb_vecs<2, VE>(st, x);
+    }
+    for (; v < nvec; v += nthreads) {
         float x[VE];
         Vec<T>::load(body + v * VE, x);
         absorb_vec(st, x);

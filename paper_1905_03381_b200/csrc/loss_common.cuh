@@ -61,6 +61,32 @@ __device__ __forceinline__ void absorb_vec(RunState& st, const float (&x)[N]) {
     st.s += a0 + a1;
 }
 
+// K vectors at once: one maximum, one comparison with the running maximum and one reference for all of them (the
+// per-vector bookkeeping is a quarter of the instructions of a bf16 vector).
+template <int K, int N>
+__device__ __forceinline__ void absorb_vecs(RunState& st, const float (&x)[K][N]) {
+    float xmax = x[0][0];
+#pragma unroll
+    for (int k = 0; k < K; ++k)
+#pragma unroll
+        for (int e = 0; e < N; ++e) xmax = fmaxf(xmax, x[k][e]);
+    const float vmax = xmax * kLog2e;
+    if (vmax > st.m) {
+        st.s *= ex2_approx(st.m - vmax);   // st.m = -inf gives 0 * 0
+        st.m = vmax;
+    }
+    const float neg_ref = st.m == -INFINITY ? 0.0f : -st.m;
+    float a0 = 0.0f, a1 = 0.0f;
+#pragma unroll
+    for (int k = 0; k < K; ++k)
+#pragma unroll
+        for (int e = 0; e < N; e += 2) {
+            a0 += ex2_approx(fmaf(x[k][e], kLog2e, neg_ref));
+            a1 += ex2_approx(fmaf(x[k][e + 1], kLog2e, neg_ref));
+        }
+    st.s += a0 + a1;
+}
+
 __device__ __forceinline__ RunState merge(const RunState& a, const RunState& b) {
     RunState o;
     o.m = fmaxf(a.m, b.m);
