@@ -148,9 +148,9 @@ __global__ void __launch_bounds__(256) row_loss_short_kernel(LossParams p) {
     }
 }
 
-// Long rows: one CTA per row.
+// Long rows: one CTA per row.  Six CTAs per SM (40 registers: the four-vector trips would take 48 and leave five).
 template <typename T>
-__global__ void __launch_bounds__(kRowThreads) row_loss_cta_kernel(LossParams p) {
+__global__ void __launch_bounds__(kRowThreads, 6) row_loss_cta_kernel(LossParams p) {
     __shared__ RunState warp_state[kRowThreads / 32];
     const int64_t rows = effective_rows(p);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
