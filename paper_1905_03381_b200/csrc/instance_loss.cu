@@ -152,27 +152,45 @@ __global__ void __launch_bounds__(256) row_loss_short_kernel(LossParams p) {
 template <typename T>
 __global__ void __launch_bounds__(kRowThreads, 6) row_loss_cta_kernel(LossParams p) {
     __shared__ RunState warp_state[kRowThreads / 32];
+    __shared__ unsigned int s_row[2];
     const int64_t rows = effective_rows(p);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
+    // Rows are handed out by the ticket counter (the first row of a CTA is its block index, the request for the row
+    // after next is in flight while a row is scanned), so that CTAs finish within one row of each other.
+    if (threadIdx.x == 0) {
+        s_row[0] = blockIdx.x;
+        s_row[1] = gridDim.x + atomicAdd(&p.ctl->ticket, 1u);
+    }
+    __syncthreads();
+    for (int it = 0;; ++it) {
+        const int64_t r = s_row[it & 1];
+        if (r >= rows) break;
+        unsigned int fresh = 0;
+        if (threadIdx.x == 0) fresh = gridDim.x + atomicAdd(&p.ctl->ticket, 1u);
         const int64_t src = source_row(p, r);                 // uniform over the CTA
         const int y = src >= 0 ? checked_label(p, src) : -1;
-        if (y < 0) {
-            if (threadIdx.x == 0) p.out[r] = 0.0f;
-            continue;
-        }
-        const T* row = static_cast<const T*>(p.logits) + src * p.row_stride;
+        const T* row = static_cast<const T*>(p.logits) + (src >= 0 ? src : 0) * p.row_stride;
         RunState st = {-INFINITY, 0.0f};
-        scan_row<T>(st, row, p.cols, threadIdx.x, kRowThreads);
+        if (y >= 0) scan_row<T>(st, row, p.cols, threadIdx.x, kRowThreads);
         st = group_merge<32>(st);
         if (lane == 0) warp_state[warp] = st;
-        __syncthreads();
+        __syncthreads();                       // every thread has read this iteration's slot of s_row
+        if (threadIdx.x == 0) s_row[it & 1] = fresh;
         if (warp == 0) {
             RunState t = lane < kRowThreads / 32 ? warp_state[lane] : RunState{-INFINITY, 0.0f};
             t = group_merge<32>(t);
-            if (lane == 0) p.out[r] = finish_row(t, Vec<T>::one(row + y));
+            if (lane == 0) p.out[r] = y >= 0 ? finish_row(t, Vec<T>::one(row + y)) : 0.0f;
         }
         __syncthreads();
+    }
+    // last CTA out re-arms the ticket counter for the next kernel on this context
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const unsigned int prev = atomicAdd(&p.ctl->done, 1u);
+        if (prev == gridDim.x - 1) {
+            p.ctl->ticket = 0;
+            p.ctl->done = 0;
+        }
     }
 }
 
