@@ -57,7 +57,7 @@ __device__ __forceinline__ void scan_row(RunState& st, const T* row, int64_t col
 
 // Short rows: LPR lanes per row, several rows per warp.
 template <typename T, int LPR>
-__global__ void __launch_bounds__(256) row_loss_group_kernel(LossParams p) {
+__global__ void __launch_bounds__(256, sizeof(T) == 4 ? 6 : 4) row_loss_group_kernel(LossParams p) {
     const int64_t rows = effective_rows(p);
     const int gl = threadIdx.x % LPR;
     const int64_t groups_per_grid = (int64_t)gridDim.x * (blockDim.x / LPR);
