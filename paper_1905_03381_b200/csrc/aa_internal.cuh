@@ -251,7 +251,6 @@ aa_status launch_shrink_from_scores(aa_ctx_impl* c, const float* score, ShrinkPa
 
 // Bulk-copy variant for 16-byte aligned rows (writes p.out); AA_ERR_UNSUPPORTED when the shape does not fit.
 struct LossParams;
-aa_status launch_instance_loss_tma(aa_ctx_impl* c, const LossParams& p, int dtype);
 
 aa_status launch_batch_cut(aa_ctx_impl* c, const int32_t* idx, const int32_t* count_dev, int64_t m_host, int64_t n_cand,
                            int64_t n_stored, int64_t batch_size, const int32_t* lengths, int64_t token_budget, int32_t* out_m,

@@ -225,7 +225,10 @@ aa_status launch_rows(aa_ctx_impl* c, LossParams& p) {
     void* args[] = {&p};
     const void* kernel;
     int threads, grid;
-    if (row_bytes >= 8 * 1024) {
+    // Up to 32 KB a warp (or part of one) owns a row: no CTA barrier per row, and with four vectors per trip that beats
+    // both a CTA per row and a bulk-copy ring with consumer warps (which this library had for 4-16 KB rows: 5.1-5.5 TB/s
+    // against 5.6-6.8 here).  Longer rows take a CTA each.
+    if (row_bytes > 32 * 1024) {
         const bool many = p.rows >= 4ll * (1536 / kRowThreadsMany) * c->sm_count;
         kernel = many ? (const void*)row_loss_cta_kernel<T, kRowThreadsMany> : (const void*)row_loss_cta_kernel<T, kRowThreads>;
         threads = many ? kRowThreadsMany : kRowThreads;
@@ -283,8 +286,7 @@ aa_status launch_instance_loss(aa_ctx_impl* c, const aa_logits& lg, const int32_
     p.ctl = c->ctl;
     p.out = offsets ? c->row_scratch : out_loss;
     if (p.rows > 0) {
-        aa_status st = row_idx ? AA_ERR_UNSUPPORTED : launch_instance_loss_tma(c, p, lg.dtype);   // the ring streams adjacent rows
-        if (st == AA_ERR_UNSUPPORTED) st = lg.dtype == AA_BF16 ? launch_rows<uint16_t>(c, p) : launch_rows<float>(c, p);
+        const aa_status st = lg.dtype == AA_BF16 ? launch_rows<uint16_t>(c, p) : launch_rows<float>(c, p);
         if (st != AA_OK) return st;
     }
     if (offsets && n_seg > 0) {

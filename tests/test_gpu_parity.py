@@ -313,8 +313,8 @@ def test_row_losses(aa, rows, cols, dtype, std):
     (34001, 1000, torch.float32, 0), (17003, 4096, torch.bfloat16, 0), (33000, 1000, torch.float32, 24),
     (140000, 512, torch.bfloat16, 0), (350001, 100, torch.float32, 0),
 ])
-def test_row_losses_large_enough_for_the_bulk_copy_kernel(aa, rows, cols, dtype, pad):
-    """128 MB and more of aligned logit rows of up to 16 KB take the bulk-copy ring kernel."""
+def test_row_losses_on_large_inputs(aa, rows, cols, dtype, pad):
+    """128 MB and more of logit rows of 0.4 to 8 KB: many rounds per CTA, strided rows, a device row count."""
     buf = W.normal((rows, cols + pad), 3.0, rows + cols, dtype, DEV)
     logits = buf[:, :cols]
     labels = W.randint(0, cols, (rows,), rows * 3 + cols, DEV)
