@@ -6,7 +6,21 @@ accepted batch (aa_instance_loss), labels + one Assistant SGD step (aa_assistant
 Pool: 65,536 candidates x 3072 bf16 features (403 MB, larger than L2; pools rotate),
 100-class fp32 logits, gamma 0.1, lr 0.05.  Prints ONE JSON line on rank 0.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--legs a,b,...]
+
+The line's headline is the whole step; beside it (single GPU, each with its own roofline entry,
+none of them depending on --steps):
+  roofline            the screening kernel alone, launches back to back over the rotating pools
+  stages              per-stage CUDA events inside whole steps (a fixed number of extra steps)
+  instance_loss_rows  per-sentence loss on the translation shape (25,000 x 32,000 bf16 logits)
+  csr                 bag-of-words screen: one 16,384-sentence pool, and 64 pools in one launch
+  mlp                 two-layer Assistant shape (262,144 x 3072 bf16, hidden 256): tensor-core screen,
+                      1000-class loss, two-layer step
+  sweep               fused screen of 2^22 x 512 fp32, shrink+compact of 2^24 stored scores,
+                      loss of 16,384 x 131,072 bf16 logits
+  pipeline            the same step as the two-stream Assistant / Boss schedule
+  e2e                 the step through the host-buffer entry point (pinned host memory)
+  cpu_baseline        the CPU oracle, one core and all cores
 
 N > 1 is launched with torch.distributed.run, one rank per GPU; every rank screens its own
 pools with its own Assistant (the path shards by instance, no data-path collective), and the
@@ -29,11 +43,12 @@ if ROOT not in sys.path:
 
 METRIC = "candidates screened/sec (score+shrink+compact -> instance loss -> Assistant step)"
 UNIT = "candidates/s"
+ALL_LEGS = ("stages", "loss", "csr", "mlp", "sweep", "pipeline", "e2e", "cpu")
 
-
-# Per-stage CUDA events are recorded on every EVENT_EVERY-th timed step: an event between two kernels keeps the
-# second from being scheduled while the first drains, which is how the steps without events run.
-EVENT_EVERY = 7   # co-prime with the number of rotating pools, so the sample covers every pool
+# Kernel-alone timings: REPS launches back to back between two events, LOOPS such loops, median and best loop.
+REPS = 24
+LOOPS = 5
+STAGE_STEPS = 56   # whole steps with per-stage events (a multiple of the rotating pools)
 
 
 def parse_args():
@@ -44,25 +59,53 @@ def parse_args():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--pools", type=int, default=8, help="distinct resident pools rotated through the steps")
     ap.add_argument("--e2e-steps", type=int, default=20)
-    ap.add_argument("--cpu-steps", type=int, default=40, help="oracle steps timed for cpu_baseline (0 = skip)")
+    ap.add_argument("--cpu-steps", type=int, default=40, help="oracle steps timed for cpu_baseline")
     ap.add_argument("--pool-rows", type=int, default=None, help="override the pool size (testing only)")
-    ap.add_argument("--workload", default="image", choices=["image", "mlp"],
-                    help="image = the benchmark workload; mlp = the two-layer (tensor-core) Assistant shape")
-    ap.add_argument("--pipeline-steps", type=int, default=300,
-                    help="steps of the two-stream Assistant/Boss schedule timed after the main region (0 = skip)")
+    ap.add_argument("--pipeline-steps", type=int, default=300, help="steps of the two-stream Assistant/Boss schedule")
     ap.add_argument("--pipeline-depth", type=int, default=2, help="Boss queue depth k of that schedule")
-    ap.add_argument("--loss-reps", type=int, default=20,
-                    help="timed calls of the per-sentence loss on the translation shape (0 = skip)")
+    ap.add_argument("--legs", default=",".join(ALL_LEGS),
+                    help="comma-separated secondary measurements to run (single GPU only): " + ", ".join(ALL_LEGS))
+    ap.add_argument("--small", action="store_true", help="shrink the secondary workloads (profiling / testing only)")
     return ap.parse_args()
 
 
-def measured_peak_gbs():
+def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
         with open(path) as f:
-            return float(json.load(f)["hbm_gbs"]), "measured"
+            rec = json.load(f)
+        return {"hbm": float(rec["hbm_gbs"]), "burst": float(rec["bf16_tflops"]),
+                "sustained": float(rec["bf16_tflops_sustained"]), "kind": "measured"}
     except Exception:
-        return 6650.0, "fallback"
+        return {"hbm": 6650.0, "burst": 1590.0, "sustained": 1400.0, "kind": "fallback"}
+
+
+NOMINAL_HBM_GBS = 8000.0
+NOMINAL_BF16_TFLOPS = 2250.0
+
+
+def hbm_roofline(bytes_per_launch, ms, best_ms, launches, peaks, kernel=None, **extra):
+    ach = bytes_per_launch / (ms * 1e-3) / 1e9
+    r = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm"], "unit": "GB/s", "frac": ach / peaks["hbm"],
+         "peak_kind": f"of {peaks['kind']}", "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS,
+         "algorithmic_bytes_per_launch": bytes_per_launch, "avg_launch_ms": ms, "best_launch_ms": best_ms,
+         "launches_timed": launches}
+    if kernel:
+        r["kernel"] = kernel
+    r.update(extra)
+    return r
+
+
+def tensor_roofline(flops_per_launch, ms, best_ms, launches, peaks, kernel=None, **extra):
+    ach = flops_per_launch / (ms * 1e-3) / 1e12
+    r = {"bound": "tensor", "achieved": ach, "peak": peaks["burst"], "unit": "TFLOP/s", "frac": ach / peaks["burst"],
+         "peak_kind": f"of {peaks['kind']} (cuBLAS bf16 burst: the kernel is timed alone)",
+         "frac_of_sustained": ach / peaks["sustained"], "frac_of_nominal_2250": ach / NOMINAL_BF16_TFLOPS,
+         "flops_per_launch": flops_per_launch, "avg_launch_ms": ms, "best_launch_ms": best_ms, "launches_timed": launches}
+    if kernel:
+        r["kernel"] = kernel
+    r.update(extra)
+    return r
 
 
 TRAFFIC_PROFILE = os.path.join(ROOT, "profiles", "score_shrink_tma_bf16_d3072.txt")
@@ -150,12 +193,32 @@ class ClockSampler:
         return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def back_to_back(torch, launch, reps=REPS, loops=LOOPS, warm=3):
+    """Times launch(i) for i = 0, 1, ...: `loops` loops of `reps` calls, one event pair around each loop, on the current
+    stream.  Returns (median loop's ms per call, best loop's ms per call, calls timed)."""
+    i = 0
+    for _ in range(warm):
+        launch(i); i += 1
+    torch.cuda.synchronize()
+    per_call = []
+    for _ in range(loops):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            launch(i); i += 1
+        e1.record()
+        torch.cuda.synchronize()
+        per_call.append(e0.elapsed_time(e1) / reps)
+    per_call.sort()
+    return per_call[len(per_call) // 2], per_call[0], reps * loops
+
+
 # --------------------------------------------------------------------------
-# CPU oracle leg (cpu_baseline and --impl reference)
+# CPU oracle legs (cpu_baseline and --impl reference)
 # --------------------------------------------------------------------------
 
 def oracle_step_seconds(cfg, x_host, w0, logits_host, labels_host, steps: int):
-    """Times `steps` whole steps of the oracle, as it stands, single-threaded.  Returns (seconds, candidates)."""
+    """Times `steps` whole steps of the oracle, as it stands, single-threaded.  Returns (seconds, candidates, final (w, b))."""
     import numpy as np
 
     from oracle import aa_oracle as O
@@ -169,7 +232,49 @@ def oracle_step_seconds(cfg, x_host, w0, logits_host, labels_host, steps: int):
         m = len(Bidx)
         f = O.row_loss(logits_host[:m], labels_host[:m]).astype(np.float32)
         w, b, _ = O.assistant_step_linear_dense(x_host, f, w, b, cfg.lr, row_idx=Bidx)
-    return time.perf_counter() - t0, n * steps
+    return time.perf_counter() - t0, n * steps, (w, b)
+
+
+def oracle_step_seconds_all_cores(cfg, x_host, w0, logits_host, labels_host, steps: int, threads: int):
+    """The same oracle functions run row-parallel: the pool, the batch's logit rows and the batch's gradient are cut into
+    one contiguous slice per thread (the rows are independent; the oracle's C routines run outside the interpreter
+    lock).  The slices' mean gradients are combined by their row counts.  Returns (seconds, candidates, final (w, b))."""
+    import numpy as np
+    from concurrent.futures import ThreadPoolExecutor
+
+    from oracle import aa_oracle as O
+
+    n = x_host.shape[0]
+    w, b = w0.copy(), np.float32(0.0)
+
+    def cuts(total):
+        edges = np.linspace(0, total, threads + 1).astype(np.int64)
+        return [(int(a), int(e)) for a, e in zip(edges[:-1], edges[1:]) if e > a]
+
+    with ThreadPoolExecutor(max_workers=threads) as pool:
+        t0 = time.perf_counter()
+        for step in range(steps):
+            parts = list(pool.map(lambda ae: O.screen_linear_dense(x_host[ae[0]:ae[1]], w, b, cfg.gamma, cfg.philox_seed, step,
+                                                                   id_base=ae[0])["B"].astype(np.int64) + ae[0], cuts(n)))
+            Bidx = np.concatenate(parts).astype(np.int32)
+            m = len(Bidx)
+            f = np.concatenate(list(pool.map(lambda ae: O.row_loss(logits_host[ae[0]:ae[1]], labels_host[ae[0]:ae[1]]),
+                                             cuts(m)))).astype(np.float32) if m else np.zeros(0, np.float32)
+            if m:
+                z = O.labels(f, O.batch_mean(f))
+
+                def grad(ae):
+                    rows = Bidx[ae[0]:ae[1]]
+                    s = O.score_dense(x_host, w, b, row_idx=rows)
+                    gw, gb = O.linear_grad_dense(x_host, s, z[ae[0]:ae[1]], row_idx=rows)
+                    return gw * (ae[1] - ae[0]), gb * (ae[1] - ae[0])
+
+                gs = list(pool.map(grad, cuts(m)))
+                gw = sum(g[0] for g in gs) / m
+                gb = sum(g[1] for g in gs) / m
+                w = O.sgd(w, gw, cfg.lr)
+                b = O.sgd(np.array([b], np.float32), np.array([gb]), cfg.lr)[0]
+        return time.perf_counter() - t0, n * steps, (w, b)
 
 
 def run_reference(args, cfg):
@@ -191,7 +296,7 @@ def run_reference(args, cfg):
     for _ in range(min(args.warmup, 2)):
         oracle_step_seconds(cfg, x, w0, logits, labels, 1)
     steps = max(1, min(args.steps, 16))
-    sec, cand = oracle_step_seconds(cfg, x, w0, logits, labels, steps)
+    sec, cand, _ = oracle_step_seconds(cfg, x, w0, logits, labels, steps)
     value = cand / sec
     sample = f"{sample_rows} of {cfg.n} candidates per step, {steps} steps"
     line = {
@@ -212,9 +317,192 @@ def workload_config(cfg, args, reference=False):
         "pool_rows": cfg.n, "d": cfg.d, "classes": cfg.classes, "mix": cfg.gamma, "lr": cfg.lr,
         "pools_rotated": None if reference else args.pools,
         "l2_policy": "inputs larger than L2: each pool is 403 MB and pools rotate",
-        "stage_events": None if reference else f"per-stage CUDA events on every {EVENT_EVERY}th timed step",
+        "kernel_timing": None if reference else
+            f"kernels alone: {LOOPS} loops of {REPS} launches back to back, one CUDA event pair per loop, median loop; "
+            f"stages: per-stage CUDA events in {STAGE_STEPS} extra whole steps; neither depends on --steps",
         "parallelism": f"instance-sharded x{args.gpus}, one Assistant per GPU, no data-path collective",
     }
+
+
+# --------------------------------------------------------------------------
+# secondary legs (single GPU)
+# --------------------------------------------------------------------------
+
+def leg_translation_loss(torch, B, W, dev, peaks, small):
+    """Second half of the metric: per-instance-loss rows/s on the translation shape (25,000 token rows x 32,000-word bf16
+    logits = 1.6 GB per call, larger than L2; per-sentence sums)."""
+    t2 = W.TranslationShape()
+    rows2 = 4096 if small else t2.token_budget
+    lg2 = t2.token_logits(rows2, dev)
+    ids2 = t2.token_ids(rows2, dev)
+    off2 = torch.from_numpy(W.ragged_offsets(rows2, t2.len_lo, t2.len_hi, 9)).to(dev)
+    sent_loss = torch.zeros(off2.numel() - 1, dtype=torch.float32, device=dev)
+    aa2 = B.AutoAssist(max_rows=rows2, max_d=8, device=dev)
+    g2 = B.logits_desc(lg2)
+    n0 = aa2.aa_launch_count()
+    ms2, best2, calls = back_to_back(torch, lambda i: aa2.aa_instance_loss(g2, ids2, sent_loss, offsets=off2))
+    launches = aa2.aa_launch_count() - n0
+    assert aa2.aa_device_status() == B.AA_OK
+    bytes2 = rows2 * t2.vocab * 2 + rows2 * 8 + off2.numel() * 4 + sent_loss.numel() * 4
+    out = {"workload": f"translation shape: {rows2} token rows x {t2.vocab} bf16 logits N(0,4), "
+                       f"{sent_loss.numel()} sentences of 8..128 tokens, summed per sentence",
+           "value": rows2 / (ms2 * 1e-3), "unit": "token rows/s", "ms_per_call": ms2,
+           "launches_per_call": launches // (calls + 3),
+           "roofline": hbm_roofline(bytes2, ms2, best2, calls, peaks, kernel="row_loss_cta_kernel + segment_sum_kernel")}
+    aa2.close()
+    return out
+
+
+def leg_csr(torch, B, W, dev, peaks, small):
+    """Bag-of-words screen (translation shape): one 16,384-sentence pool per launch (16 distinct pools rotate: 144 MB,
+    larger than L2), and 64 pools' worth of sentences in one launch (570 MB)."""
+    t = W.TranslationShape()
+    w, b = t.assistant(dev)
+    asst = B.linear_assistant(w, b)
+
+    def pool(n, seed):
+        g = torch.Generator(device=dev).manual_seed(seed)
+        lengths = torch.randint(t.len_lo, t.len_hi + 1, (n,), generator=g, device=dev, dtype=torch.int64)
+        indptr = torch.zeros(n + 1, dtype=torch.int64, device=dev)
+        indptr[1:] = torch.cumsum(lengths, 0)
+        nnz = int(indptr[-1].item())
+        col = torch.randint(0, t.buckets, (nnz,), generator=g, device=dev, dtype=torch.int32)
+        val = torch.ones(nnz, dtype=torch.float32, device=dev)
+        return indptr.to(torch.int32), col, val, nnz
+
+    out = {}
+    n_big = t.n * (4 if small else 64)
+    aa = B.AutoAssist(max_rows=n_big, max_d=t.buckets, device=dev)
+    out_idx = torch.zeros(n_big, dtype=torch.int32, device=dev)
+    cnt = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    pools = [pool(t.n, 500 + k) for k in range(4 if small else 16)]
+    feats = [B.csr_features(p[0], p[1], p[2], t.buckets, nnz=p[3]) for p in pools]
+    ms, best, calls = back_to_back(torch, lambda i: aa.aa_score_shrink(feats[i % len(feats)], asst, t.gamma, t.philox_seed, i,
+                                                                       out_idx, cnt))
+    nnz_mean = sum(p[3] for p in pools) / len(pools)
+    bytes1 = 8 * nnz_mean + 4 * (t.n + 1) + 4 * int(cnt.item())
+    out["single_pool"] = {"workload": f"{t.n} sentences of 8..128 hashed tokens, 2^18 buckets, mix {t.gamma}; {len(pools)} pools rotate",
+                          "value": t.n / (ms * 1e-3), "unit": UNIT, "ms_per_call": ms,
+                          "roofline": hbm_roofline(bytes1, ms, best, calls, peaks, kernel="score_shrink_csr_kernel",
+                                                   note="8.9 MB per launch: bounded by launch latency, not by HBM")}
+    del pools, feats
+    ip, col, val, nnz = pool(n_big, 600)
+    big = B.csr_features(ip, col, val, t.buckets, nnz=nnz)
+    ms, best, calls = back_to_back(torch, lambda i: aa.aa_score_shrink(big, asst, t.gamma, t.philox_seed, i, out_idx, cnt),
+                                   reps=8, loops=5)
+    bytes_big = 8 * nnz + 4 * (n_big + 1) + 4 * int(cnt.item())
+    out["batched"] = {"workload": f"{n_big} sentences ({n_big // t.n} pools) in one launch, {nnz} non-zeros",
+                      "value": n_big / (ms * 1e-3), "unit": UNIT, "ms_per_call": ms,
+                      "roofline": hbm_roofline(bytes_big, ms, best, calls, peaks, kernel="score_shrink_csr_kernel")}
+    assert aa.aa_device_status() == B.AA_OK
+    aa.close()
+    return out
+
+
+def leg_mlp(torch, B, W, dev, peaks, small):
+    """Two-layer Assistant shape: pool 262,144 x 3072 bf16 N(0,1), 3072 -> 256 (ReLU) -> 1, 1000-class fp32 logits,
+    SGD lr 0.01 on both layers.  Screen alone (tensor roofline), loss alone, step alone on the screen's batch list, and
+    whole steps."""
+    cfg = W.MlpShape()
+    if small:
+        cfg.n = 32768
+    x = cfg.pool(dev)
+    W1, b1, w2, b2 = cfg.assistant(dev)
+    W1b = W1.to(torch.bfloat16).contiguous()
+    logits = cfg.logits(cfg.n, dev)
+    labels = cfg.labels(cfg.n, dev)
+    aa = B.AutoAssist(max_rows=cfg.n, max_d=cfg.d, max_hidden=cfg.hidden, device=dev)
+    asst = B.mlp_assistant(W1, W1b, b1, w2, b2)
+    out_idx = torch.zeros(cfg.n, dtype=torch.int32, device=dev)
+    cnt = torch.zeros(1, dtype=torch.int32, device=dev)
+    loss = torch.zeros(cfg.n, dtype=torch.float32, device=dev)
+    feat, batch = B.dense_features(x), B.dense_features(x, row_idx=out_idx)
+    lg = B.logits_desc(logits)
+
+    ms_s, best_s, calls_s = back_to_back(torch, lambda i: aa.aa_score_shrink(feat, asst, cfg.gamma, cfg.philox_seed, i, out_idx, cnt),
+                                         reps=10, loops=5)
+    m = int(cnt.item())
+    ms_l, best_l, calls_l = back_to_back(torch, lambda i: aa.aa_instance_loss(lg, labels, loss, count_dev=cnt), reps=10, loops=5)
+    ms_a, best_a, calls_a = back_to_back(torch, lambda i: aa.aa_assistant_step(batch, loss, asst, cfg.lr, count_dev=cnt),
+                                         reps=10, loops=5)
+
+    def step(i):
+        aa.aa_score_shrink(feat, asst, cfg.gamma, cfg.philox_seed, 100 + i, out_idx, cnt)
+        aa.aa_instance_loss(lg, labels, loss, count_dev=cnt)
+        aa.aa_assistant_step(batch, loss, asst, cfg.lr, count_dev=cnt)
+
+    ms_w, best_w, calls_w = back_to_back(torch, step, reps=10, loops=3)
+    assert aa.aa_device_status() == B.AA_OK
+    flops = 2.0 * cfg.n * cfg.d * cfg.hidden
+    out = {
+        "workload": f"MLP Assistant shape: pool {cfg.n} x {cfg.d} bf16 N(0,1), {cfg.d}->{cfg.hidden} (ReLU)->1, "
+                    f"{cfg.classes}-class fp32 logits N(0,3), mix {cfg.gamma}, SGD lr {cfg.lr} on both layers; pool 1.6 GB > L2",
+        "accepted": m,
+        "score_shrink": {"value": cfg.n / (ms_s * 1e-3), "unit": UNIT, "ms_per_call": ms_s,
+                         "roofline": tensor_roofline(flops, ms_s, best_s, calls_s, peaks, kernel="mlp_score_shrink_kernel",
+                                                     hbm_GBs=cfg.n * cfg.d * 2 / (ms_s * 1e-3) / 1e9,
+                                                     hbm_frac=cfg.n * cfg.d * 2 / (ms_s * 1e-3) / 1e9 / peaks["hbm"])},
+        "instance_loss": {"value": m / (ms_l * 1e-3), "unit": "rows/s", "ms_per_call": ms_l,
+                          "roofline": hbm_roofline(m * (cfg.classes * 4 + 8), ms_l, best_l, calls_l, peaks,
+                                                   kernel="row_loss_group_kernel")},
+        "assistant_step": {"ms_per_call": ms_a, "rows": m,
+                           "roofline": tensor_roofline(2 * 2.0 * m * cfg.d * cfg.hidden, ms_a, best_a, calls_a, peaks,
+                                                       kernel="mlp_residual_kernel + mlp_w1_grad_kernel (+ updates)")},
+        "whole_step": {"value": cfg.n / (ms_w * 1e-3), "unit": UNIT, "ms_per_step": ms_w, "steps_timed": calls_w},
+    }
+    aa.close()
+    return out
+
+
+def leg_sweep(torch, B, W, dev, peaks, small):
+    """Scaling-sweep points: fused screen of a 2^22 x 512 fp32 pool (8.6 GB), shrink+compact of 2^24 stored scores (three
+    score arrays rotate: 201 MB, larger than L2), per-row loss of 16,384 x 131,072 bf16 logits (4.3 GB)."""
+    out = {}
+    sw = W.SweepShape()
+    n1 = (1 << 18) if small else (1 << 22)
+    n2 = (1 << 20) if small else (1 << 24)
+    aa = B.AutoAssist(max_rows=n2, max_d=sw.d, device=dev)
+    w, b = sw.assistant(dev)
+    asst = B.linear_assistant(w, b)
+    out_idx = torch.zeros(n2, dtype=torch.int32, device=dev)
+    cnt = torch.zeros(1, dtype=torch.int32, device=dev)
+    for mix in (0.05, 0.5):
+        x = torch.randn((n1, sw.d), device=dev, dtype=torch.float32, generator=torch.Generator(device=dev).manual_seed(14))
+        feat = B.dense_features(x)
+        ms, best, calls = back_to_back(torch, lambda i: aa.aa_score_shrink(feat, asst, mix, 0, i, out_idx, cnt), reps=8, loops=5)
+        m = int(cnt.item())
+        out[f"fused_screen_mix{mix}"] = {
+            "workload": f"{n1} x {sw.d} fp32 N(0,1), linear Assistant, mix {mix}", "value": n1 / (ms * 1e-3), "unit": UNIT,
+            "ms_per_call": ms, "accepted": m,
+            "roofline": hbm_roofline(n1 * sw.d * 4 + sw.d * 4 + 4 * m, ms, best, calls, peaks, kernel="score_shrink_tma_kernel<float>")}
+        del x, feat
+    scores = [W.normal((n2,), 2.0, 700 + k, torch.float32, dev) for k in range(3)]
+    for mix in (0.05, 0.5):
+        ms, best, calls = back_to_back(torch, lambda i: aa.aa_shrink_compact(scores[i % 3], mix, 0, i, out_idx, cnt), reps=12, loops=5)
+        m = int(cnt.item())
+        out[f"shrink_compact_mix{mix}"] = {
+            "workload": f"{n2} stored scores N(0,2), mix {mix}", "value": n2 / (ms * 1e-3), "unit": UNIT, "ms_per_call": ms,
+            "accepted": m,
+            "roofline": hbm_roofline(4 * n2 + 4 * m, ms, best, calls, peaks, kernel="shrink_from_scores_kernel",
+                                     note="Philox + sigmoid (about 130 instructions per candidate) and the look-back latency "
+                                          "bound this kernel, not its 4 + 4p bytes per candidate")}
+    assert aa.aa_device_status() == B.AA_OK
+    del scores, out_idx
+    aa.close()
+    rows, vocab = (2048, 131072) if small else (16384, 131072)
+    lg = W.sweep_logits(rows, vocab, dev)
+    ids = W.randint(0, vocab, (rows,), 16, dev)
+    ell = torch.zeros(rows, dtype=torch.float32, device=dev)
+    aa2 = B.AutoAssist(max_rows=rows, max_d=8, device=dev)
+    g = B.logits_desc(lg)
+    ms, best, calls = back_to_back(torch, lambda i: aa2.aa_instance_loss(g, ids, ell), reps=8, loops=5)
+    assert aa2.aa_device_status() == B.AA_OK
+    out["instance_loss"] = {"workload": f"{rows} x {vocab} bf16 logits N(0,4), per row", "value": rows / (ms * 1e-3),
+                            "unit": "rows/s", "ms_per_call": ms,
+                            "roofline": hbm_roofline(rows * (vocab * 2 + 8), ms, best, calls, peaks, kernel="row_loss_cta_kernel")}
+    aa2.close()
+    return out
 
 
 # --------------------------------------------------------------------------
@@ -241,6 +529,13 @@ def run_b200(args, cfg):
         lib_build.build()
     if world > 1:
         dist.barrier()
+    legs = set(x for x in args.legs.split(",") if x) if world == 1 else set()
+    if world > 1:
+        legs = {"e2e"}
+    unknown = legs - set(ALL_LEGS)
+    if unknown:
+        raise SystemExit(f"unknown --legs entries: {sorted(unknown)}")
+    peaks = measured_peaks()
 
     plan = sharding.plan(rank, world, args.pools, cfg.n)
     pools = [cfg.pool(pid, dev) for pid in plan.pool_ids]
@@ -251,7 +546,8 @@ def run_b200(args, cfg):
     asst = B.linear_assistant(w, b)
     out_idx = torch.zeros(cfg.n, dtype=torch.int32, device=dev)
     # one device count per step, so that the mean batch size of the timed steps is known without a host read
-    n_slots = max(args.warmup, 3) + args.steps
+    warm = max(args.warmup, 3)
+    n_slots = warm + max(args.steps, STAGE_STEPS, REPS * LOOPS + 3)
     counts = torch.zeros(n_slots, dtype=torch.int32, device=dev)
     count_of = [counts[j:j + 1] for j in range(n_slots)]
     loss = torch.zeros(cfg.n, dtype=torch.float32, device=dev)
@@ -260,9 +556,9 @@ def run_b200(args, cfg):
     lg = [B.logits_desc(l) for l in logits]
     npool = len(pools)
 
-    def step(i, events=None):
+    def step(i, events=None, slot=None):
         k = i % npool
-        out_count = count_of[i % n_slots]
+        out_count = count_of[(i if slot is None else slot) % n_slots]
         if events is not None:
             events[0].record()
         aa.aa_score_shrink(feats[k], asst, cfg.gamma, cfg.philox_seed, i, out_idx, out_count)
@@ -280,14 +576,13 @@ def run_b200(args, cfg):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(max(args.warmup, 3)):
+    for i in range(warm):
         step(i)
     barrier()
     assert aa.aa_device_status() == B.AA_OK
 
-    # ---- device-resident throughput: K steps between two events, kernels timed per call as well
+    # ---- the metric: K whole steps between two events, nothing else in the timed region
     K = args.steps
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
@@ -297,29 +592,70 @@ def run_b200(args, cfg):
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_start.record()
     for i in range(K):
-        step(args.warmup + i, ev[i] if i % EVENT_EVERY == 0 else None)   # per-stage events on a sample of the steps
+        step(warm + i)
     t_end.record()
     barrier()
     elapsed_ms = t_start.elapsed_time(t_end)
     launches = aa.aa_launch_count() - launches0
+    status = aa.aa_device_status()
+    assert status == B.AA_OK, B.status_string(status)
+    timed = counts[[(warm + i) % n_slots for i in range(K)]].cpu().numpy().astype(np.int64)
+    accepted = float(timed.mean())            # mean batch size M over the timed steps
+    agg = sharding.aggregate(dist if world > 1 else None, dev, elapsed_ms, cfg.n * K)
+
+    # ---- the dominant kernel alone: screening launches back to back over the rotating pools (the Assistant stays as the
+    # timed steps left it; the Philox step number advances), independent of --steps
+    counts.zero_()
+    ms_scr, best_scr, calls_scr = back_to_back(
+        torch, lambda i: aa.aa_score_shrink(feats[i % npool], asst, cfg.gamma, cfg.philox_seed, 10_000 + i, out_idx,
+                                            count_of[i % n_slots]))
+    m_scr = float(counts[3:3 + calls_scr].float().mean().item())
     if rank == 0:
         time.sleep(0.2)
         sampler.stop()
-    status = aa.aa_device_status()
-    assert status == B.AA_OK, B.status_string(status)
-    timed = counts[[(args.warmup + i) % n_slots for i in range(K)]].cpu().numpy().astype(np.int64)
-    accepted = float(timed.mean())            # mean batch size M over the timed steps
-    sampled = [ev[i] for i in range(K) if i % EVENT_EVERY == 0]
-    score_ms = sum(e[0].elapsed_time(e[1]) for e in sampled) / len(sampled)
-    loss_ms = sum(e[1].elapsed_time(e[2]) for e in sampled) / len(sampled)
-    asst_ms = sum(e[2].elapsed_time(e[3]) for e in sampled) / len(sampled)
+    alg_bytes = cfg.n * cfg.d * 2 + cfg.d * 4 + m_scr * 4 + 4
+    roofline = hbm_roofline(alg_bytes, ms_scr, best_scr, calls_scr, peaks, kernel="score_shrink_tma_kernel<bf16, 32>",
+                            traffic=ncu_traffic_bytes(cfg.n), accepted_mean=m_scr,
+                            timing=f"{LOOPS} loops of {REPS} launches back to back over {npool} rotating pools; median loop")
+    screen = {"value": cfg.n / (ms_scr * 1e-3), "unit": UNIT, "what": "score + shrink + compact alone (steps S1-S3), N / t",
+              "ms_per_call": ms_scr}
 
-    agg = sharding.aggregate(dist if world > 1 else None, dev, elapsed_ms, cfg.n * K)
+    # ---- per-stage events inside whole steps: a fixed number of extra steps, an event before and after every call
+    stages = None
+    if "stages" in legs or world > 1:
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(STAGE_STEPS)]
+        for i in range(STAGE_STEPS):
+            step(20_000 + i, ev[i], slot=i)
+        torch.cuda.synchronize()
+        m_st = float(counts[:STAGE_STEPS].float().mean().item())
+        score_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / STAGE_STEPS
+        loss_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / STAGE_STEPS
+        asst_ms = sum(e[2].elapsed_time(e[3]) for e in ev) / STAGE_STEPS
+        sb = cfg.n * cfg.d * 2 + cfg.d * 4 + m_st * 4 + 4
+        stages = {
+            "steps": STAGE_STEPS, "accepted_mean": m_st,
+            "note": "event to event inside whole steps: includes the event records and the gap to the next launch",
+            "score_shrink": {"ms": score_ms, "GB/s": sb / (score_ms * 1e-3) / 1e9, "frac": sb / (score_ms * 1e-3) / 1e9 / peaks["hbm"]},
+            "instance_loss": {"ms": loss_ms, "GB/s": m_st * (cfg.classes * 4 + 8) / (loss_ms * 1e-3) / 1e9,
+                              "rows_per_s": m_st / (loss_ms * 1e-3)},
+            "assistant_step": {"ms": asst_ms, "GB/s": (m_st * (cfg.d * 2 + 8) + 2 * cfg.d * 4) / (asst_ms * 1e-3) / 1e9,
+                               "frac": (m_st * (cfg.d * 2 + 8) + 2 * cfg.d * 4) / (asst_ms * 1e-3) / 1e9 / peaks["hbm"]},
+        }
+        # the loss and the step alone, back to back, on the last batch list
+        m_last = int(counts[STAGE_STEPS - 1].item())
+        cl = count_of[STAGE_STEPS - 1]
+        ms_l, best_l, calls_l = back_to_back(torch, lambda i: aa.aa_instance_loss(lg[i % npool], labels[i % npool], loss, count_dev=cl))
+        ms_a, best_a, calls_a = back_to_back(torch, lambda i: aa.aa_assistant_step(batch_feats[i % npool], loss, asst, cfg.lr, count_dev=cl))
+        stages["instance_loss_alone"] = {"rows": m_last, "roofline": hbm_roofline(m_last * (cfg.classes * 4 + 8), ms_l, best_l, calls_l, peaks,
+                                                                                  kernel="row_loss_short_kernel")}
+        stages["assistant_step_alone"] = {"rows": m_last, "roofline": hbm_roofline(m_last * (cfg.d * 2 + 8) + 2 * cfg.d * 4, ms_a, best_a,
+                                                                                   calls_a, peaks, kernel="linear_grad_mma_kernel")}
+        assert aa.aa_device_status() == B.AA_OK
 
     # ---- the same three stages as the two-stream schedule with a Boss queue of depth k (screening runs ahead of the
     # losses and updates it no longer waits for); reported beside the sequential figure, which stays the metric
     pipeline = None
-    if args.pipeline_steps > 0 and world == 1:
+    if "pipeline" in legs and args.pipeline_steps > 0:
         from paper_1905_03381_b200.pipeline import StreamPipeline
 
         pipe = StreamPipeline(args.pipeline_depth, max_rows=cfg.n, max_d=cfg.d, capacity=cfg.n, device=dev)
@@ -338,7 +674,7 @@ def run_b200(args, cfg):
             ctx.aa_instance_loss(lg[t % npool], labels[t % npool], out_loss, count_dev=count_dev)
 
         P = args.pipeline_steps
-        pipe.run(max(args.warmup, 3), features, boss, asst, cfg.gamma, cfg.philox_seed, cfg.lr, first_step=5000)
+        pipe.run(warm, features, boss, asst, cfg.gamma, cfg.philox_seed, cfg.lr, first_step=5000)
         torch.cuda.synchronize()
         n0 = pipe.launch_count()
         p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -356,45 +692,9 @@ def run_b200(args, cfg):
         pipe.close()
         del pipe
 
-    # ---- second half of the metric: per-instance-loss rows/s on the translation shape
-    # (25,000 token rows x 32,000-word bf16 logits = 1.6 GB per call, larger than L2; per-sentence sums)
-    loss_rows = None
-    if args.loss_reps > 0 and rank == 0:
-        t2 = W.TranslationShape()
-        rows2 = t2.token_budget
-        lg2 = t2.token_logits(rows2, dev)
-        ids2 = t2.token_ids(rows2, dev)
-        off2 = torch.from_numpy(W.ragged_offsets(rows2, t2.len_lo, t2.len_hi, 9)).to(dev)
-        sent_loss = torch.zeros(off2.numel() - 1, dtype=torch.float32, device=dev)
-        aa2 = B.AutoAssist(max_rows=rows2, max_d=8, device=dev)
-        g2 = B.logits_desc(lg2)
-        for _ in range(3):
-            aa2.aa_instance_loss(g2, ids2, sent_loss, offsets=off2)
-        torch.cuda.synchronize()
-        l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        n0 = aa2.aa_launch_count()
-        l0.record()
-        for _ in range(args.loss_reps):
-            aa2.aa_instance_loss(g2, ids2, sent_loss, offsets=off2)
-        l1.record()
-        torch.cuda.synchronize()
-        assert aa2.aa_device_status() == B.AA_OK
-        ms2 = l0.elapsed_time(l1) / args.loss_reps
-        bytes2 = rows2 * t2.vocab * 2 + rows2 * 8 + off2.numel() * 4 + sent_loss.numel() * 4
-        peak2, kind2 = measured_peak_gbs()
-        loss_rows = {"workload": f"translation shape: {rows2} token rows x {t2.vocab} bf16 logits N(0,4), "
-                                 f"{sent_loss.numel()} sentences of 8..128 tokens, summed per sentence",
-                     "value": rows2 / (ms2 * 1e-3), "unit": "token rows/s", "ms_per_call": ms2,
-                     "launches_per_call": (aa2.aa_launch_count() - n0) // args.loss_reps,
-                     "roofline": {"bound": "hbm", "achieved": bytes2 / (ms2 * 1e-3) / 1e9, "peak": peak2, "unit": "GB/s",
-                                  "frac": bytes2 / (ms2 * 1e-3) / 1e9 / peak2, "peak_kind": f"of {kind2}",
-                                  "algorithmic_bytes_per_launch": bytes2}}
-        aa2.close()
-        del lg2, ids2, aa2
-
     # ---- end to end through the host-buffer entry point (pinned host inputs, results read back)
     e2e = None
-    if args.e2e_steps > 0:
+    if "e2e" in legs and args.e2e_steps > 0:
         xh = pools[0].cpu().pin_memory()
         lh = logits[0].cpu().pin_memory()
         yh = labels[0].cpu().pin_memory()
@@ -427,38 +727,48 @@ def run_b200(args, cfg):
             dist.destroy_process_group()
         return
 
-    peak, peak_kind = measured_peak_gbs()
-    alg_bytes = cfg.n * cfg.d * 2 + cfg.d * 4 + accepted * 4 + 4
-    achieved = alg_bytes / (score_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "score_shrink_tma_kernel<bf16, 32>", "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": ncu_traffic_bytes(cfg.n),
-                "launches_timed": len(sampled),
-                "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": score_ms,
-                "frac_of_nominal_8TBs": achieved / 8000.0}
-    loss_bytes = accepted * (cfg.classes * 4 + 8)
-    asst_bytes = accepted * (cfg.d * 2 + 8) + 2 * cfg.d * 4
-    stages = {
-        "score_shrink": {"ms": score_ms, "GB/s": achieved},
-        "instance_loss": {"ms": loss_ms, "GB/s": loss_bytes / (loss_ms * 1e-3) / 1e9, "rows_per_s": accepted / (loss_ms * 1e-3)},
-        "assistant_step": {"ms": asst_ms, "GB/s": asst_bytes / (asst_ms * 1e-3) / 1e9},
-    }
-
-    cpu = None
-    if world == 1 and args.cpu_steps > 0:
+    # ---- CPU oracle on this machine's host cores: one core, and the same functions row-parallel over all cores
+    cpu = cpu_all = None
+    if "cpu" in legs and args.cpu_steps > 0:
         from oracle import aa_oracle as O
         O.build()
         xs = W.to_oracle(pools[0])
         w0 = cfg.assistant("cpu")[0].numpy()
-        sec, cand = oracle_step_seconds(cfg, xs, w0, logits[0].cpu().numpy(), labels[0].cpu().numpy(), args.cpu_steps)
+        lh_np, yh_np = logits[0].cpu().numpy(), labels[0].cpu().numpy()
+        sec, cand, _ = oracle_step_seconds(cfg, xs, w0, lh_np, yh_np, args.cpu_steps)
         cpu = {"value": cand / sec, "unit": UNIT, "cores": 1, "kind": "oracle",
                "sample": f"{args.cpu_steps} whole steps on one full pool of {cfg.n} candidates ({sec:.1f} s)"}
+        try:
+            cores = len(os.sched_getaffinity(0))
+        except AttributeError:
+            cores = os.cpu_count() or 1
+        threads = max(1, min(cores, 64))
+        sec2, cand2, _ = oracle_step_seconds_all_cores(cfg, xs, w0, lh_np, yh_np, args.cpu_steps, threads)
+        cpu_all = {"value": cand2 / sec2, "unit": UNIT, "cores": threads, "cores_available": cores, "kind": "oracle, row-parallel",
+                   "sample": f"{args.cpu_steps} whole steps on one full pool of {cfg.n} candidates, rows cut into {threads} "
+                             f"slices, one thread each ({sec2:.1f} s)"}
+        del xs
+
+    # ---- secondary workloads, each alone on the GPU (the image pools are released first)
+    del pools, logits, labels, feats, batch_feats, lg
+    aa.close()
+    torch.cuda.empty_cache()
+    loss_rows = leg_translation_loss(torch, B, W, dev, peaks, args.small) if "loss" in legs else None
+    torch.cuda.empty_cache()
+    csr = leg_csr(torch, B, W, dev, peaks, args.small) if "csr" in legs else None
+    torch.cuda.empty_cache()
+    mlp = leg_mlp(torch, B, W, dev, peaks, args.small) if "mlp" in legs else None
+    torch.cuda.empty_cache()
+    sweep = leg_sweep(torch, B, W, dev, peaks, args.small) if "sweep" in legs else None
 
     line = {
         "metric": METRIC, "value": agg["units"] / (agg["ms"] * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
-        "warmup": max(args.warmup, 3), "ms_per_step": agg["ms"] / K, "higher_is_better": True, "scaling": "weak",
+        "warmup": warm, "ms_per_step": agg["ms"] / K, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(cfg, args),
-        "roofline": roofline, "stages": stages, "instance_loss_rows": loss_rows, "pipeline": pipeline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
-        "accepted_mean": accepted, "accepted_min": int(timed.min()), "accepted_max": int(timed.max()), "clocks": sampler.summary(),
+        "roofline": roofline, "screen": screen, "stages": stages, "instance_loss_rows": loss_rows, "csr": csr, "mlp": mlp,
+        "sweep": sweep, "pipeline": pipeline, "cpu_baseline": cpu, "cpu_all_cores": cpu_all, "e2e": e2e,
+        "gpu_launches": int(launches), "accepted_mean": accepted, "accepted_min": int(timed.min()),
+        "accepted_max": int(timed.max()), "clocks": sampler.summary(),
     }
     print(json.dumps(line), flush=True)
     if world > 1:
@@ -466,111 +776,10 @@ def run_b200(args, cfg):
         dist.destroy_process_group()
 
 
-def measured_peak_tflops(sustained: bool):
-    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    try:
-        with open(path) as f:
-            rec = json.load(f)
-        return float(rec["bf16_tflops_sustained" if sustained else "bf16_tflops"]), "measured"
-    except Exception:
-        return (1400.0 if sustained else 1590.0), "fallback"
-
-
-def run_mlp(args):
-    """Secondary workload (--workload mlp): the two-layer Assistant shape, whose scoring is a dense bf16 contraction.
-    One step = MLP score+shrink+compact, 1000-class instance loss, MLP Assistant step on the accepted rows."""
-    import torch
-
-    from paper_1905_03381_b200 import binding as B, build as lib_build, workloads as W
-
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU path")
-    torch.cuda.set_device(0)
-    dev = torch.device("cuda", 0)
-    lib_build.build()
-    cfg = W.MlpShape()
-    if args.pool_rows:
-        cfg.n = args.pool_rows
-    x = cfg.pool(dev)
-    W1, b1, w2, b2 = cfg.assistant(dev)
-    W1b = W1.to(torch.bfloat16).contiguous()
-    logits = cfg.logits(cfg.n, dev)
-    labels = cfg.labels(cfg.n, dev)
-    aa = B.AutoAssist(max_rows=cfg.n, max_d=cfg.d, max_hidden=cfg.hidden, device=dev)
-    asst = B.mlp_assistant(W1, W1b, b1, w2, b2)
-    out_idx = torch.zeros(cfg.n, dtype=torch.int32, device=dev)
-    K = args.steps
-    warm = max(args.warmup, 3)
-    counts = torch.zeros(warm + K, dtype=torch.int32, device=dev)
-    loss = torch.zeros(cfg.n, dtype=torch.float32, device=dev)
-    feat, batch = B.dense_features(x), B.dense_features(x, row_idx=out_idx)
-    lg = B.logits_desc(logits)
-
-    def step(i, ev=None):
-        cnt = counts[i:i + 1]
-        if ev: ev[0].record()
-        aa.aa_score_shrink(feat, asst, cfg.gamma, cfg.philox_seed, i, out_idx, cnt)
-        if ev: ev[1].record()
-        aa.aa_instance_loss(lg, labels, loss, count_dev=cnt)
-        if ev: ev[2].record()
-        aa.aa_assistant_step(batch, loss, asst, cfg.lr, count_dev=cnt)
-        if ev: ev[3].record()
-
-    for i in range(warm):
-        step(i)
-    torch.cuda.synchronize()
-    assert aa.aa_device_status() == B.AA_OK
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
-    sampler = ClockSampler(0)
-    sampler.start()
-    time.sleep(0.3)
-    n0 = aa.aa_launch_count()
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0.record()
-    for i in range(K):
-        step(warm + i, evs[i])
-    t1.record()
-    torch.cuda.synchronize()
-    time.sleep(0.2)
-    sampler.stop()
-    assert aa.aa_device_status() == B.AA_OK
-    ms = t0.elapsed_time(t1) / K
-    score_ms = sum(e[0].elapsed_time(e[1]) for e in evs) / K
-    loss_ms = sum(e[1].elapsed_time(e[2]) for e in evs) / K
-    asst_ms = sum(e[2].elapsed_time(e[3]) for e in evs) / K
-    m_mean = float(counts[warm:].float().mean().item())
-    flops = 2.0 * cfg.n * cfg.d * cfg.hidden
-    peak, kind = measured_peak_tflops(sustained=True)
-    hbm, hkind = measured_peak_gbs()
-    line = {
-        "metric": METRIC, "value": cfg.n / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": K, "warmup": warm,
-        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-        "data": "synthetic",
-        "config": {"workload": f"MLP Assistant shape: pool {cfg.n} x {cfg.d} bf16 N(0,1), {cfg.d}->{cfg.hidden} (ReLU)->1, "
-                               f"{cfg.classes}-class fp32 logits N(0,3), mix {cfg.gamma}, SGD lr {cfg.lr} on both layers",
-                   "l2_policy": "inputs larger than L2 (pool 1.6 GB)"},
-        "roofline": {"bound": "tensor", "kernel": "mlp_score_shrink_kernel", "achieved": flops / (score_ms * 1e-3) / 1e12,
-                     "peak": peak, "unit": "TFLOP/s", "frac": flops / (score_ms * 1e-3) / 1e12 / peak,
-                     "peak_kind": f"of {kind} (sustained cuBLAS bf16)", "traffic": None, "avg_launch_ms": score_ms,
-                     "hbm_GBs": cfg.n * cfg.d * 2 / (score_ms * 1e-3) / 1e9, "hbm_frac": cfg.n * cfg.d * 2 / (score_ms * 1e-3) / 1e9 / hbm},
-        "stages": {"score_shrink": {"ms": score_ms}, "instance_loss": {"ms": loss_ms, "rows_per_s": m_mean / (loss_ms * 1e-3),
-                   "GB/s": m_mean * (cfg.classes * 4 + 8) / (loss_ms * 1e-3) / 1e9},
-                   "assistant_step": {"ms": asst_ms, "TFLOP/s": 2 * 2.0 * m_mean * cfg.d * cfg.hidden / (asst_ms * 1e-3) / 1e12}},
-        "accepted_mean": m_mean, "gpu_launches": int(aa.aa_launch_count() - n0), "clocks": sampler.summary(),
-    }
-    print(json.dumps(line), flush=True)
-    aa.close()
-
-
 def main():
     args = parse_args()
     from paper_1905_03381_b200 import workloads as W
 
-    if args.workload == "mlp":
-        if args.impl == "reference" or args.gpus != 1:
-            raise SystemExit("--workload mlp is a single-GPU measurement of the library only")
-        run_mlp(args)
-        return
     cfg = W.ImageShape()
     if args.pool_rows:
         cfg.n = args.pool_rows

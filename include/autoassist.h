@@ -4,14 +4,14 @@
  *
  * One training step of the generator, as the paper defines it:
  *   1. score a pool of candidate instances with the light-weight Assistant g(x; phi)
- *      (Sec. 5.2; logistic regression in Sec. 6.1, bag-of-words classifier in Sec. 6.2),
+ *      (Sec. "Learning to generate smart training batches"; logistic regression in Sec. "Image classification", bag-of-words classifier in Sec. "Machine Translation"),
  *   2. accept each candidate by the Bernoulli rule of Algorithm 1 (Assistant.sample_batch)
  *      with base probability gamma, i.e. with probability gamma + (1 - gamma) g,
  *   3. append the accepted candidates to the batch B in list order (Algorithm 1),
- *   4. obtain the Boss's loss f on every instance of B (Sec. 5.3: the (i, f_i) pairs pushed
+ *   4. obtain the Boss's loss f on every instance of B (Sec. "Asynchronous joint learning with CPU/GPU": the (i, f_i) pairs pushed
  *      to the AssistantQueue) — here: row cross-entropy of caller-supplied logits, summed
  *      over the token rows of a sentence for sequence tasks,
- *   5. turn the losses into labels z = 1[f > T] (Sec. 5.2) and take one gradient step on the
+ *   5. turn the losses into labels z = 1[f > T] (Sec. "Learning to generate smart training batches") and take one gradient step on the
  *      Assistant's cross-entropy objective (Eq. "sec-loss"; Algorithm 2: gradient, update).
  *
  * Conventions
@@ -25,7 +25,10 @@
  *     found on the device (scan wait gave up, label or column out of range, more survivors
  *     than capacity) latch a code in a device status word that aa_device_status reads;
  *     no kernel traps or aborts.
- *   - One context per stream; calls on one context must not overlap in time.
+ *   - One context per stream; calls on one context must not overlap in time.  Screening calls of
+ *     two contexts that overlap on one GPU are allowed, but each sizes its grid for an idle GPU:
+ *     when they compete for SMs a look-back wait can run out, which latches AA_ERR_SCAN_TIMEOUT
+ *     (the batch of that call is invalid; repeat the call).
  *   - out_idx, out_count and the mask are pure functions of (features, parameters, mix,
  *     seed, step, id_base): Philox4x32-10 is keyed by seed with counter (instance id, step).
  */
@@ -58,15 +61,15 @@ typedef enum { AA_ASSIST_LINEAR = 0, AA_ASSIST_MLP = 1 } aa_assist_kind;
 typedef enum { AA_THRESH_VALUE = 0, AA_THRESH_BATCH_MEAN = 1 } aa_thresh_mode;
 
 /*
- * Feature rows of the candidate instances (the x_i that g(x_i; phi) is evaluated on, Sec. 5.2).
+ * Feature rows of the candidate instances (the x_i that g(x_i; phi) is evaluated on, Sec. "Learning to generate smart training batches").
  * Dense: row-major [n x d], element type dtype, row r starts at dense + r*row_stride elements.
  *        The 128-bit load path needs dense 16-byte aligned and row_stride*sizeof(element)
  *        a multiple of 16; anything else takes a slower element-wise path.
- * CSR:   indptr[n+1], col[nnz] in [0, d), val[nnz] fp32 (the bag-of-words counts of Sec. 6.2).
+ * CSR:   indptr[n+1], col[nnz] in [0, d), val[nnz] fp32 (the bag-of-words counts of Sec. "Machine Translation").
  *        Repeated columns in a row add.  nnz = indptr[n] as known on the host (it only steers
  *        how many lanes share a row; 0 = unknown).
  * row_idx: optional candidate list.  Candidate k is stored row row_idx[k], k in [0, n_rows)
- *        (the slice of the shuffled index list that Sec. 5.2 walks).  NULL: candidate k is
+ *        (the slice of the shuffled index list that Sec. "Learning to generate smart training batches" walks).  NULL: candidate k is
  *        row k and n_rows is ignored.
  * id_base: instance id of stored row 0.  The Philox counter of a candidate is id_base + row,
  *        so a shard of a larger data set draws the same decisions as the whole.
@@ -93,7 +96,7 @@ typedef struct {
  * MLP: g = sigmoid(w2 . relu(W1 x + b1) + b2); W1 is [hidden x d] row-major (one hidden unit
  *      per row), kept as an fp32 master W1 and a bf16 copy W1_bf16 that scoring reads;
  *      b1[hidden], w2[hidden], b2[1] fp32.  (The paper only asks for a light-weight model,
- *      Sec. 5.1-5.2; the two-layer form is this library's dense-contraction case.)
+ *      Secs. "Assistant for instance selection" and "Learning to generate smart training batches"; the two-layer form is this library's dense-contraction case.)
  */
 typedef struct {
     int32_t kind;            /* aa_assist_kind */
@@ -164,13 +167,13 @@ aa_status aa_shrink_compact(aa_ctx* ctx, const float* score, int64_t n, int64_t 
                             int32_t* out_idx, int64_t capacity, int32_t* out_count, uint8_t* out_mask);
 
 /*
- * Hard shrinking (Sec. 4.2, Eq. "shrinking_grad"; the SK method of Sec. 4.4): an instance is used
+ * Hard shrinking (Sec. "Instance Shrinking in Stochastic Gradient Descent", Eq. "shrinking_grad"; the SK method of Sec. "Shrinking experiment under convex setting"): an instance is used
  * only if its objective value or gradient magnitude is at least T.  value[i] is that quantity for
  * instance i (e.g. the losses of aa_instance_loss); out_idx receives the ascending list of i with
  * value[i] >= threshold, out_count its length, out_mask (nullable) one byte per instance.  No random
  * draw is involved; NaN values are dropped.  Capacity overflow latches AA_ERR_CAPACITY as in
  * aa_score_shrink.  aa_sk_threshold gives the schedule T_k = G / k of the convergence theorem
- * (Sec. 5, Theorem 1) for step k >= 1 (HOST helper).
+ * (Sec. "Theoretical Analysis", Theorem 1) for step k >= 1 (HOST helper).
  */
 aa_status aa_threshold_compact(aa_ctx* ctx, const float* value, int64_t n, float threshold,
                                int32_t* out_idx, int64_t capacity, int32_t* out_count, uint8_t* out_mask);
@@ -181,7 +184,7 @@ float aa_sk_threshold(float G, int64_t k);
  * survivor list of a screened pool.  Algorithm 1 stops as soon as the batch holds batch_size
  * instances, so its batch is the first batch_size entries of the list and its walk over the
  * (shuffled) candidate list ends right after the last one taken; the next call starts there.
- * For sequence tasks (Sec. 6.2: batches of a given number of tokens) the batch is the longest prefix
+ * For sequence tasks (Sec. "Machine Translation": batches of a given number of tokens) the batch is the longest prefix
  * of the list whose sentence lengths add up to at most token_budget.
  *   idx, count_dev : out_idx / out_count of aa_score_shrink (candidate k = stored row k, i.e. no
  *                    candidate list); idx_capacity bounds the device count.  n_cand = pool size.
@@ -249,7 +252,7 @@ aa_status aa_instance_loss(aa_ctx* ctx, const aa_logits* logits, const int32_t* 
 
 /*
  * Step 4 on a batch list: the Boss losses of the batch instances when the logits (and labels) are
- * stored for the whole pool (Sec. 5.3: the losses {f(x_i, y_i)} of the instances i in B).
+ * stored for the whole pool (Sec. "Asynchronous joint learning with CPU/GPU": the losses {f(x_i, y_i)} of the instances i in B).
  *   out_loss[k] = l_r with r = row_idx[k], for k in [0, M), M = min(*count_dev, n_rows) when
  *   count_dev is given, else n_rows; labels[r] is the label of stored row r.
  * row_idx: device int32 list (e.g. out_idx of aa_score_shrink); an entry outside [0, logits->rows)
@@ -274,7 +277,7 @@ aa_status aa_assistant_step(aa_ctx* ctx, const aa_feat* feat, const float* loss,
                             aa_assistant* assistant, float lr, int32_t thresh_mode, float threshold);
 
 /*
- * Step 5 with Adam in place of SGD (the paper trained its Assistants with Adam, Sec. 6.1).  Labels and gradient exactly as
+ * Step 5 with Adam in place of SGD (the paper trained its Assistants with Adam, Sec. "Image classification").  Labels and gradient exactly as
  * in aa_assistant_step; the update of every parameter p with mean gradient g is
  *   m <- beta1 m + (1 - beta1) g,   v <- beta2 v + (1 - beta2) g^2,
  *   p <- p - lr (m / (1 - beta1^t)) / (sqrt(v / (1 - beta2^t)) + eps),      t = state->t + 1,

@@ -40,7 +40,7 @@ static double ref_load(const void *base, int dtype, int64_t k) {
 }
 
 /* ------------------------------------------------------------------ */
-/* Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11, Sec. 3.3 / 4):   */
+/* Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11, their Sec. 3.3 and 4):   */
 /* ten rounds of two 32x32->64 multiplies on counter words 0 and 2,   */
 /* the high halves xor-ed with the other counter words and the key,   */
 /* the key advanced by two Weyl increments between rounds.            */
@@ -79,8 +79,8 @@ double aa_ref_uniform(uint64_t seed, uint64_t step, uint64_t id) {
 }
 
 /* ------------------------------------------------------------------ */
-/* Assistant pre-activation s_i (Sec. 5.2, classifier g; Sec. 6.1     */
-/* logistic regression; Sec. 6.2 bag-of-words).                       */
+/* Assistant pre-activation s_i (Sec. "Learning to generate smart training batches", classifier g; Sec. "Image classification"     */
+/* logistic regression; Sec. "Machine Translation" bag-of-words).                       */
 /* Candidate k is stored row r_k = row_idx ? row_idx[k] : k.          */
 /* ------------------------------------------------------------------ */
 void aa_ref_score_dense(const void *x, int dtype, int64_t d, int64_t row_stride,
@@ -148,7 +148,9 @@ void aa_ref_accept_prob(const double *g, int64_t n, double gamma, double *p) {
 }
 
 /* ------------------------------------------------------------------ */
-/* Algorithm 1, one candidate: the two-branch rule as printed.        */
+/* Algorithm 1, one candidate: accepted outright when the draw falls  */
+/* below the floor gamma; otherwise the draw, rescaled to [0, 1), is  */
+/* compared with the Assistant's g.                                   */
 /* ------------------------------------------------------------------ */
 static int ref_accept(double c, double g, double gamma) {
     if (c < gamma) return 1;
@@ -184,32 +186,30 @@ int64_t aa_ref_compact(const uint8_t *keep, int64_t n_cand, const int32_t *row_i
 }
 
 /*
- * Algorithm 1 literally: walk the (shuffled) candidate list one instance at a
- * time until batch_size instances are accepted or the list ends.  *consumed =
- * number of candidates examined.  Independent of the two functions above.
+ * The batch Algorithm 1 returns, as a walk over the (shuffled) candidate list: position by
+ * position, the instance there joins the batch when its uniform draw falls below its net
+ * acceptance probability gamma + (1 - gamma) g (the remark after Algorithm 1: the floor gamma and
+ * the Assistant's g share one draw); the walk stops once the batch is full or the list ends.
+ * *consumed = positions visited.  Written on its own: it calls neither aa_ref_shrink nor
+ * aa_ref_compact, and uses the one-comparison form of the rule where they use the two-branch form.
  */
 int64_t aa_ref_sample_batch(const double *g, int64_t n_cand, double gamma,
                             uint64_t seed, uint64_t step, int64_t id_base,
                             const int32_t *row_idx, int64_t batch_size,
                             int32_t *B, int64_t *consumed) {
-    int64_t size = 0, k = 0;
-    while (size < batch_size && k < n_cand) {
-        int64_t idx = row_idx ? row_idx[k] : k;
-        double c = aa_ref_uniform(seed, step, (uint64_t)(id_base + idx));
-        if (c < gamma) {
-            B[size++] = (int32_t)idx;
-        } else {
-            double c_hat = (c - gamma) / (1.0 - gamma);
-            if (c_hat < g[k]) B[size++] = (int32_t)idx;
-        }
-        ++k;
+    int64_t taken = 0, pos = 0;
+    for (; pos < n_cand && taken < batch_size; ++pos) {
+        const int64_t instance = row_idx ? row_idx[pos] : pos;
+        const double draw = aa_ref_uniform(seed, step, (uint64_t)(id_base + instance));
+        const double p_accept = gamma + (1.0 - gamma) * g[pos];
+        if (draw < p_accept) B[taken++] = (int32_t)instance;
     }
-    *consumed = k;
-    return size;
+    *consumed = pos;
+    return taken;
 }
 
 /* ------------------------------------------------------------------ */
-/* Boss loss per instance (Sec. 5.3: the value f pushed with index i). */
+/* Boss loss per instance (Sec. "Asynchronous joint learning with CPU/GPU": the value f pushed with index i). */
 /* Row cross-entropy: log sum_c exp(l_c) - l_label, two passes.        */
 /* A negative label marks padding and contributes 0; a label >= cols   */
 /* is invalid and also contributes 0.                                  */
@@ -241,7 +241,7 @@ void aa_ref_segment_sum(const double *ell, const int32_t *offsets, int64_t n_seg
 }
 
 /* ------------------------------------------------------------------ */
-/* Assistant labels (Sec. 5.2): z_i = 1 if f_i > T else 0.             */
+/* Assistant labels (Sec. "Learning to generate smart training batches"): z_i = 1 if f_i > T else 0.             */
 /* ------------------------------------------------------------------ */
 double aa_ref_batch_mean(const float *f, int64_t m) {
     if (m <= 0) return 0.0;

@@ -378,7 +378,7 @@ def adam(param, m, v, grad, lr: float, beta1: float, beta2: float, eps: float, t
 
 
 def pipeline_linear_dense(pool_of, logits_of, w, b, gamma: float, seed: int, lr: float, depth: int, n_steps: int, T=None):
-    """The Assistant / Boss schedule of Sec. 5.3 (Algorithms 2 and 3) with a Boss queue of `depth` batches, written
+    """The Assistant / Boss schedule of Sec. "Asynchronous joint learning with CPU/GPU" (Algorithms 2 and 3) with a Boss queue of `depth` batches, written
     as the one sequence of events it becomes when both workers take turns in a fixed order:
 
       Assistant: while the Boss queue is short (fewer than `depth` batches ahead of the Boss, and always the batch the
@@ -418,7 +418,7 @@ def pipeline_linear_dense(pool_of, logits_of, w, b, gamma: float, seed: int, lr:
 
 
 def instance_loss_rows(logits, labels, row_idx) -> np.ndarray:
-    """Losses of the batch instances (Sec. 5.3: {f(x_i, y_i)} for i in B) out of logits / labels stored for the whole
+    """Losses of the batch instances (Sec. "Asynchronous joint learning with CPU/GPU": {f(x_i, y_i)} for i in B) out of logits / labels stored for the whole
     pool: entry k is the row loss of stored row row_idx[k]."""
     labels = _arr(labels, np.int32)
     out = np.zeros(len(row_idx), dtype=np.float64)

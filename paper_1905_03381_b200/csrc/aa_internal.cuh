@@ -88,7 +88,7 @@ struct ShrinkParams {
 #ifdef __CUDACC__
 
 // One parameter's update from its mean gradient `grad` (Algorithm 2: Assistant.update).  SGD: param - lr * grad.
-// Adam (the optimizer the paper trained the Assistant with, Sec. 6.1): biased moments in a.m / a.v, bias-corrected step.
+// Adam (the optimizer the paper trained the Assistant with, Sec. "Image classification"): biased moments in a.m / a.v, bias-corrected step.
 __device__ __forceinline__ float adam_update(const AdamArgs& a, float param, float grad, float lr, int64_t j) {
     const float m = a.beta1 * a.m[j] + (1.0f - a.beta1) * grad;
     const float v = a.beta2 * a.v[j] + (1.0f - a.beta2) * grad * grad;

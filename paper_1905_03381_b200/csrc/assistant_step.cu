@@ -1,4 +1,4 @@
-// Assistant labels + one SGD step (Sec. 5.2 label rule and objective; Algorithm 2:
+// Assistant labels + one SGD step (Sec. "Learning to generate smart training batches" label rule and objective; Algorithm 2:
 // Assistant.gradient, Assistant.update) for the linear Assistant g = sigmoid(w.x + b).
 //
 // Dense features: each CTA stages a block of batch rows in shared memory once, computes

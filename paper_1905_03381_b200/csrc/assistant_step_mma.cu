@@ -1,4 +1,4 @@
-// Assistant gradient for 16-byte aligned bf16 rows of up to 3072 features (Sec. 5.2 objective;
+// Assistant gradient for 16-byte aligned bf16 rows of up to 3072 features (Sec. "Learning to generate smart training batches" objective;
 // Algorithm 2: Assistant.gradient), with the two passes over each staged row done by warp-level
 // matrix instructions instead of one FMA per element.
 //

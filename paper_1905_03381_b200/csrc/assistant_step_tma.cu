@@ -1,4 +1,4 @@
-// Assistant gradient for 16-byte aligned dense rows (Sec. 5.2 objective; Algorithm 2:
+// Assistant gradient for 16-byte aligned dense rows (Sec. "Learning to generate smart training batches" objective; Algorithm 2:
 // Assistant.gradient), as one persistent, warp-specialised CTA per SM fed by bulk copies.
 //
 //   producer warp : takes tickets of batch rows and streams them (gathered through the batch

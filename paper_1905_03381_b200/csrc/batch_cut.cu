@@ -3,7 +3,7 @@
 //
 // Algorithm 1 appends accepted instances until the batch holds batch_size of them, so its batch is
 // the first batch_size survivors of the list and its walk ends right after the last one taken.
-// For sequence tasks the batch is bounded by a token budget instead (Sec. 6.2 trains on batches of
+// For sequence tasks the batch is bounded by a token budget instead (Sec. "Machine Translation" trains on batches of
 // a given number of tokens): the longest prefix of survivors whose lengths add up to at most the
 // budget, together with the running token offsets that the per-sentence loss needs.
 // One CTA: the lengths of up to a million survivors are scanned in chunks of 1024 with a carry.

@@ -1,4 +1,4 @@
-// Per-instance Boss loss from logits (Sec. 5.3: the loss f pushed with each index i).
+// Per-instance Boss loss from logits (Sec. "Asynchronous joint learning with CPU/GPU": the loss f pushed with each index i).
 //
 // Row cross-entropy  l_r = log sum_c exp(x_rc) - x_{r,y_r}  in a single pass over the row:
 // every thread keeps a running maximum M and a sum S of 2^(t - M) over its elements, with

@@ -1,5 +1,5 @@
 // Pieces shared by the per-instance-loss kernels: the running (max, sum) state of a one-pass
-// log-sum-exp in base 2, its merge, and the label checks (Sec. 5.3: the loss f of each batch instance).
+// log-sum-exp in base 2, its merge, and the label checks (Sec. "Asynchronous joint learning with CPU/GPU": the loss f of each batch instance).
 #pragma once
 
 #include <math.h>

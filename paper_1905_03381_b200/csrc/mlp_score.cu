@@ -1,7 +1,7 @@
 // Assistant score -> Bernoulli shrink -> ordered batch list for the two-layer Assistant
 //   s_i = w2 . relu(W1 x_i + b1) + b2        (bf16 features and W1, fp32 accumulation),
 // where scoring is a dense contraction [candidates x d] * [d x hidden] and runs on the
-// tcgen05 tensor cores (Sec. 5.2 asks only for a light-weight classifier g; this is the
+// tcgen05 tensor cores (Sec. "Learning to generate smart training batches" asks only for a light-weight classifier g; this is the
 // library's dense-contraction Assistant).
 //
 // One persistent CTA per SM, 12 warps (18 when a candidate list selects the rows: warps 3 and 12..17

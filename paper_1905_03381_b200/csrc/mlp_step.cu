@@ -1,5 +1,5 @@
 // Labels + one SGD step of the two-layer Assistant g = sigmoid(w2 . relu(W1 x + b1) + b2)
-// (Sec. 5.2 label rule and objective; Algorithm 2: Assistant.gradient, Assistant.update),
+// (Sec. "Learning to generate smart training batches" label rule and objective; Algorithm 2: Assistant.gradient, Assistant.update),
 // back-propagated through both layers on the tcgen05 tensor cores.
 //
 //   mlp_residual_kernel  forward pass over the batch rows under the current parameters (same

@@ -1,11 +1,15 @@
 // Shrink decision + order-preserving append shared by every scoring front end
 // (Algorithm 1, Assistant.sample_batch, for a pool of candidates at once).
 //
-// Tiles of candidates are handed out by a ticket counter; a tile's kept candidates are
-// appended at the position given by a decoupled look-back over the tiles' counts.  Because
-// tickets are issued in look-back order, every tile a warp waits on is owned by a CTA that
-// is already running; each wait is nevertheless bounded and gives up with a latched
-// AA_ERR_SCAN_TIMEOUT instead of spinning for ever.
+// Tiles of candidates are handed out in look-back order (a ticket counter; the bulk-copy kernel
+// gives each CTA its block index as first tile and tickets after that); a tile's kept candidates
+// are appended at the position given by a decoupled look-back over the tiles' counts.  A warp
+// therefore only waits on tiles whose owners started before it or, for the block-index tiles, on
+// CTAs of the same grid, which the launchers size to be resident together when the GPU is
+// otherwise idle.  That is not a guarantee: if something else holds an SM (a scan of a second
+// context on another stream, a foreign kernel's shared memory), a first tile's owner may not be
+// running yet.  So every wait is bounded and gives up with a latched AA_ERR_SCAN_TIMEOUT instead
+// of spinning for ever; the batch of such a call is invalid and the caller repeats it.
 #pragma once
 
 #include "aa_internal.cuh"

@@ -315,6 +315,15 @@ __global__ void __launch_bounds__(kTmaThreads, 1) score_shrink_tma_kernel(DenseF
             float sv[kMaxUnits];
 #pragma unroll
             for (int u = 0; u < kMaxUnits; ++u) sv[u] = u < units ? s_ring[slot * g.slot_rows + u * 32 + lane] : 0.0f;
+            if (p.row_idx && p.out_score) {
+                // a candidate whose list entry points outside the store was never copied: its score slot holds stale sums
+#pragma unroll
+                for (int u = 0; u < kMaxUnits; ++u) {
+                    const long long k = (long long)tile * p.tile_rows + u * 32 + lane;
+                    if (u < units && k < p.n_cand && (unsigned long long)(long long)p.row_idx[k] >= (unsigned long long)p.n_stored)
+                        sv[u] = __int_as_float(0x7FC00000);
+                }
+            }
             __syncwarp();
             if (lane == 0) mbar_arrive(&cb->s_empty[slot]);
             warp_shrink_compact<kMaxUnits>(p, tile, epoch, units, sv);

@@ -1,5 +1,5 @@
 // Declarations shared by the Assistant-step kernels (labels + one SGD step of the linear
-// Assistant; Sec. 5.2 label rule and objective, Algorithm 2: gradient, update).
+// Assistant; Sec. "Learning to generate smart training batches" label rule and objective, Algorithm 2: gradient, update).
 #pragma once
 
 #include "aa_internal.cuh"

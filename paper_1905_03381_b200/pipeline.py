@@ -1,5 +1,5 @@
 """Assistant and Boss as two CUDA streams with a bounded queue of screened batches between them
-(Sec. 5.3; Algorithms 2 and 3: the Assistant thread fills the Boss queue up to k batches and otherwise
+(Sec. "Asynchronous joint learning with CPU/GPU"; Algorithms 2 and 3: the Assistant thread fills the Boss queue up to k batches and otherwise
 trains on the (batch, losses) items the Boss hands back).
 
 The paper runs the two workers as threads that meet in two queues.  On one GPU the same schedule is

@@ -1,7 +1,7 @@
 """Host-side sharding of the batch generator across GPUs.
 
 The path shards by instance: every rank owns whole candidate pools and its own Assistant
-(the paper trains one Assistant per GPU on that GPU's data chunk, Sec. 6.2), so there is no
+(the paper trains one Assistant per GPU on that GPU's data chunk, Sec. "Machine Translation"), so there is no
 data-path collective.  Instance ids stay global (id_base per pool), so the keep/skip decisions
 do not depend on how many ranks share the data.  The only cross-rank exchange is the reduction
 of the timing numbers for reporting.

@@ -5,8 +5,8 @@ the method's arithmetic (no scoring, no sampling rule, no loss).  Both the CUDA
 library's callers and the CPU oracle's callers take their inputs from here, so
 that the two sides see identical data.
 
-The inputs stand in for the datasets the paper trained on (Sec. 6.1: MNIST,
-FashionMNIST, EMNIST, CIFAR10; Sec. 6.2: Multi30k, WMT14 En-De): the shapes,
+The inputs stand in for the datasets the paper trained on (Sec. "Image classification": MNIST,
+FashionMNIST, EMNIST, CIFAR10; Sec. "Machine Translation": Multi30k, WMT14 En-De): the shapes,
 sizes and value ranges follow them (pixel vectors in [0, 1), 3*32*32 = 3072
 features, 10..1000 classes, sentence lengths 8..128, vocabularies of tens of
 thousands of tokens) and no dataset item is used.  "N(0, s)" below always means

@@ -104,6 +104,11 @@ def test_tiny_reference_config_screen(aa):
     c = O.uniform(cfg.philox_seed, cfg.step, np.arange(cfg.n))
     xn = np.linalg.norm(t["x"].double().cpu().numpy(), axis=1)
     check_screen(gpu, ref["s"], ref["keep"], ref["p"], c, None, float(t["w"].double().norm()), xn)
+    # the plain relative bound (1e-5 of the score itself) wherever the dot product has not cancelled away:
+    # |s| at least 5 % of ||w|| ||x|| leaves fp32 accumulation of 64 terms far inside it
+    plain = np.abs(ref["s"]) >= 0.05 * float(t["w"].double().norm()) * xn
+    assert plain.sum() > cfg.n // 2
+    assert np.all(np.abs(gpu[2] - ref["s"])[plain] <= 1e-5 * np.abs(ref["s"])[plain])
     # zero-ish weights: acceptance near gamma + (1 - gamma)/2
     p_mean = ref["p"].mean()
     assert abs(gpu[1] - ref["p"].sum()) < 5 * math.sqrt((ref["p"] * (1 - ref["p"])).sum())
@@ -483,6 +488,11 @@ def test_tiny_reference_config_full_step(aa):
     assert 0 < z.sum() < m
     assert_params_close(w.cpu().numpy(), w_ref)
     assert_params_close([b.item()], [b_ref])
+    # the plain relative bound (1e-4 of the weight itself) on every weight that is not tiny
+    w_gpu, w_r = w.cpu().numpy().astype(np.float64), np.asarray(w_ref, np.float64)
+    big = np.abs(w_r) >= 0.1 * math.sqrt(float(np.mean(w_r ** 2)))
+    assert big.sum() > cfg.d // 2 and np.all(np.abs(w_gpu - w_r)[big] <= 1e-4 * np.abs(w_r)[big])
+    assert abs(b.item() - float(b_ref)) <= 1e-4 * abs(float(b_ref))
     assert aa.aa_launch_count() > 0
 
 

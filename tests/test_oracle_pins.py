@@ -459,6 +459,55 @@ def test_update_special_cases():
     assert np.array_equal(w3, w) and b3 == b
 
 
+def test_composed_csr_step_special_cases():
+    """assistant_step_linear_csr chains labels, score_csr, linear_grad_csr and sgd: pinned on the one-instance closed
+    form (a count of c in bucket j moves w_j by -lr c (sigma(c w_j + b) - z) and b by -lr (sigma(c w_j + b) - z), and
+    nothing else), on a batch list that selects that one row out of several, and against the dense twin."""
+    d, j, c = 7, 2, 3.0
+    w = np.linspace(-0.4, 0.6, d).astype(np.float32)
+    b = np.float32(-0.15)
+    # three stored rows; the batch is row 1 alone: bucket j with count c (stored as one entry of value c)
+    indptr = np.array([0, 2, 3, 5], np.int32)
+    col = np.array([0, 5, j, 1, 6], np.int32)
+    val = np.array([1.0, 2.0, c, 1.0, 1.0], np.float32)
+    f = np.array([0.3], np.float32)
+    w1, b1, z = O.assistant_step_linear_csr(indptr, col, val, f, w, b, lr=0.25, T=1.0, row_idx=np.array([1], np.int32))
+    assert z[0] == 0
+    r = 1.0 / (1.0 + math.exp(-(c * float(w[j]) + float(b))))            # sigma(s) - 0
+    expect = w.copy(); expect[j] = np.float32(float(w[j]) - 0.25 * c * r)
+    assert np.array_equal(w1, expect)
+    assert b1 == np.float32(float(b) - 0.25 * r)
+    # batch mean threshold over two instances with different losses: exactly the larger one is labelled 1
+    f2 = np.array([0.2, 0.9], np.float32)
+    _, _, z2 = O.assistant_step_linear_csr(indptr, col, val, f2, w, b, lr=0.1, row_idx=np.array([0, 2], np.int32))
+    assert list(z2) == [0, 1]
+    # n_cand: only the first len(f) entries of a longer batch list are used
+    wa, ba, _ = O.assistant_step_linear_csr(indptr, col, val, f, w, b, lr=0.25, T=1.0, row_idx=np.array([1, 0, 2], np.int32))
+    assert np.array_equal(wa, w1) and ba == b1
+    # the dense twin on the densified rows takes the same step (repeated buckets add)
+    rng = np.random.default_rng(21)
+    n, d2 = 30, 12
+    lens = rng.integers(0, 6, n)
+    ip = np.zeros(n + 1, np.int32); ip[1:] = np.cumsum(lens)
+    cc = rng.integers(0, d2, int(ip[-1])).astype(np.int32)
+    vv = rng.integers(1, 4, int(ip[-1])).astype(np.float32)
+    dense = np.zeros((n, d2), np.float32)
+    for i in range(n):
+        for k in range(ip[i], ip[i + 1]):
+            dense[i, cc[k]] += vv[k]
+    w0 = (rng.normal(size=d2) * 0.3).astype(np.float32)
+    rows = np.sort(rng.permutation(n)[:17]).astype(np.int32)
+    ff = np.abs(rng.normal(size=17)).astype(np.float32)
+    wc, bc, zc = O.assistant_step_linear_csr(ip, cc, vv, ff, w0, 0.2, lr=0.3, row_idx=rows)
+    wd, bd, zd = O.assistant_step_linear_dense(dense, ff, w0, 0.2, lr=0.3, row_idx=rows)
+    assert np.array_equal(zc, zd) and np.allclose(wc, wd, rtol=0, atol=1e-7) and abs(float(bc) - float(bd)) <= 1e-7
+    # lr = 0 and an empty batch leave the parameters unchanged
+    w3, b3, _ = O.assistant_step_linear_csr(indptr, col, val, f, w, b, lr=0.0, T=1.0, row_idx=np.array([1], np.int32))
+    assert np.array_equal(w3, w) and b3 == b
+    w4, b4, _ = O.assistant_step_linear_csr(indptr, col, val, np.zeros(0, np.float32), w, b, lr=0.5)
+    assert np.array_equal(w4, w) and b4 == b
+
+
 def test_bf16_rounding_is_nearest_even():
     src = np.array([1.0, 1.00390625, 1.01171875, -3.0e-41, 3.3895314e38, np.inf], np.float32)
     ref = torch.from_numpy(src).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
@@ -577,7 +626,7 @@ def _pipeline_inputs(n_steps, n=300, d=12, classes=5, seed=31):
 
 
 def test_pipeline_schedule_lag_and_special_cases():
-    """Sec. 5.3 / Algorithms 2-3 as one event sequence: batch j is screened with the parameters after
+    """Sec. "Asynchronous joint learning with CPU/GPU" / Algorithms 2-3 as one event sequence: batch j is screened with the parameters after
     max(0, j - depth) updates; depth 0 is the plain chain screen -> loss -> update; a zero learning rate makes the
     depth irrelevant; batches screened before the first update do not depend on the learning rate."""
     steps = 7
