@@ -547,7 +547,7 @@ def run_b200(args, cfg):
     out_idx = torch.zeros(cfg.n, dtype=torch.int32, device=dev)
     # one device count per step, so that the mean batch size of the timed steps is known without a host read
     warm = max(args.warmup, 3)
-    n_slots = warm + max(args.steps, STAGE_STEPS, REPS * LOOPS + 3)
+    n_slots = warm + max(args.steps, STAGE_STEPS + 1, REPS * LOOPS + 3)
     counts = torch.zeros(n_slots, dtype=torch.int32, device=dev)
     count_of = [counts[j:j + 1] for j in range(n_slots)]
     loss = torch.zeros(cfg.n, dtype=torch.float32, device=dev)
@@ -641,9 +641,12 @@ def run_b200(args, cfg):
             "assistant_step": {"ms": asst_ms, "GB/s": (m_st * (cfg.d * 2 + 8) + 2 * cfg.d * 4) / (asst_ms * 1e-3) / 1e9,
                                "frac": (m_st * (cfg.d * 2 + 8) + 2 * cfg.d * 4) / (asst_ms * 1e-3) / 1e9 / peaks["hbm"]},
         }
-        # the loss and the step alone, back to back, on the last batch list
-        m_last = int(counts[STAGE_STEPS - 1].item())
-        cl = count_of[STAGE_STEPS - 1]
+        # the loss and the step alone, back to back, on the batch list of a screen under the initial Assistant
+        # (weights near zero: about gamma + (1 - gamma) / 2 of the pool, the mean batch of the steps above)
+        w_init, b_init = cfg.assistant(dev)
+        cl = count_of[STAGE_STEPS]
+        aa.aa_score_shrink(feats[0], B.linear_assistant(w_init, b_init), cfg.gamma, cfg.philox_seed, 30_000, out_idx, cl)
+        m_last = int(cl.item())
         ms_l, best_l, calls_l = back_to_back(torch, lambda i: aa.aa_instance_loss(lg[i % npool], labels[i % npool], loss, count_dev=cl))
         ms_a, best_a, calls_a = back_to_back(torch, lambda i: aa.aa_assistant_step(batch_feats[i % npool], loss, asst, cfg.lr, count_dev=cl))
         stages["instance_loss_alone"] = {"rows": m_last, "roofline": hbm_roofline(m_last * (cfg.classes * 4 + 8), ms_l, best_l, calls_l, peaks,
