@@ -6,17 +6,21 @@
 //                        TMA/MMA pipeline as scoring, but in tiles of 128 rows whose two
 //                        accumulators alternate: the passes over one tile's accumulator run
 //                        while the products of the next tile are issued), then per row  z = 1[loss > T],
-//                        r = sigmoid(s) - z,  and per hidden unit u the factor
-//                        P[i][u] = r_i [a_iu > 0]  of delta1_iu = r_i w2_u [a_iu > 0].
-//                        P is stored transposed in bf16 ([hidden x rows]); the column sums
-//                        sum_i r_i relu(a_iu) (-> grad w2), sum_i P[i][u] (-> grad b1) and
+//                        r = sigmoid(s) - z,  and per hidden unit u the gate [a_iu > 0] of
+//                        delta1_iu = r_i w2_u [a_iu > 0].  What leaves for the W1 gradient is small:
+//                        the gates as one bit each (64 rows x 256 units per 2 KB block) and r_i as
+//                        two bf16 terms r_hi + r_lo (16 mantissa bits together).  The column sums
+//                        sum_i r_i relu(a_iu) (-> grad w2), sum_i r_i [a_iu > 0] (-> grad b1) and
 //                        sum_i r_i (-> grad b2) stay in fp32 and leave as per-CTA partials.
-//   mlp_w1_grad_kernel   G[u][k] = sum_i P[i][u] x_ik : a [hidden x rows] x [rows x d] contraction
-//                        over the batch rows.  A CTA owns 256 feature columns and a slice of
-//                        the rows (split-K): per 64-row slice, P^T as a K-major operand and the
-//                        feature rows themselves as an MN-major operand (the contraction runs
-//                        down the rows, 128-byte swizzle), two [128 x 256] fp32 accumulators in
-//                        TMEM (hidden units 0..127 and 128..255).  Partials go to the workspace.
+//   mlp_w1_grad_kernel   G[u][k] = sum_i P[i][u] x_ik with P[i][u] = r_i [a_iu > 0]: a [hidden x rows] x
+//                        [rows x d] contraction over the batch rows.  A CTA owns 256 feature columns and a
+//                        slice of the rows (split-K).  Per 64-row slice the feature rows arrive by TMA as an
+//                        MN-major operand (the contraction runs down the rows, 128-byte swizzle), while eight
+//                        warps BUILD the other operand in shared memory from the gate bits and r: one
+//                        K-major [hidden x 64] bf16 tile for r_hi and one for r_lo, both multiplied into the
+//                        same two [128 x 256] fp32 accumulators in TMEM (hidden units 0..127 and 128..255).
+//                        No P matrix crosses HBM or L2, and the bf16 rounding of r (2^-9) does not reach the
+//                        gradient.  Partials go to the workspace.
 //   mlp_apply_w1_kernel  W1 <- W1 - lr (w2_u / M) sum_splits G ; W1_bf16 <- round-to-nearest-even(W1).
 //   mlp_apply_small_kernel  b1, w2, b2 from the column-sum partials (reads the old w2 first).
 #include <cuda_bf16.h>
@@ -53,8 +57,10 @@ struct MlpStepParams {
     int64_t d;
     MlpGeom g;
     // workspace
-    __nv_bfloat16* Pt;        // [hidden][pitch]
-    int64_t pitch;
+    uint32_t* gate_bits;      // [pitch / 64][kMaxHidden][2]: bit (i & 31) of word (i >> 5) & 1 = [a_iu > 0] for row i, unit u
+    __nv_bfloat16* r_hi;      // [pitch]: r_i rounded to bf16
+    __nv_bfloat16* r_lo;      // [pitch]: r_i - r_hi rounded to bf16
+    int64_t pitch;            // batch rows rounded up to whole tiles
     float* small;             // [ctas][2 * kMaxHidden + 1]: sum r relu(a), sum P, sum r
     float* part;              // [splits][hidden][d_pad]
     int64_t d_pad;
@@ -192,8 +198,14 @@ mlp_residual_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                 r = sigmoid_f32(s + bias2) - z;
             }
             sum_r += r;
-            const __nv_bfloat16 r_bf = __float2bfloat16_rn(r);
-            const __nv_bfloat16 zero_bf = __float2bfloat16_rn(0.0f);
+            {
+                // r as two bf16 terms: the W1-gradient contraction multiplies each of them with the rows
+                const __nv_bfloat16 hi = __float2bfloat16_rn(r);
+                p.r_hi[i] = hi;
+                p.r_lo[i] = __float2bfloat16_rn(r - __bfloat162float(hi));
+            }
+            // gate words of this warp's 32 rows (adjacent in i): word (i >> 5) & 1 of block i >> 6
+            uint32_t* gate_dst = p.gate_bits + (((int64_t)tile * kHalfRows + quad * 32) >> 6) * (2 * kMaxHidden) + (quad & 1);
 #pragma unroll
             for (int c = 0; c < kMaxHidden / 32; ++c) {
                 const int c0 = c * 32;
@@ -202,15 +214,17 @@ mlp_residual_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                     tmem_ld_32cols(t_row + (uint32_t)c0, a);
                     tmem_ld_wait();
                     float rh[32], pm[32];
+                    uint32_t mine = 0;
 #pragma unroll
                     for (int q = 0; q < 32; ++q) {
                         const float pre = __uint_as_float(a[q]) + b1_s[c0 + q];
                         const bool on = pre > 0.0f;
                         rh[q] = on ? r * pre : 0.0f;
                         pm[q] = on ? r : 0.0f;
-                        // P^T[u][i]: the warp's 32 rows are adjacent in i
-                        p.Pt[(int64_t)(c0 + q) * p.pitch + i] = on ? r_bf : zero_bf;
+                        const uint32_t gates = __ballot_sync(0xFFFFFFFFu, on);   // unit c0 + q over the warp's rows
+                        if (lane == q) mine = gates;
                     }
+                    gate_dst[(c0 + lane) * 2] = mine;
                     sum_rh[c] += lanes_transpose_sum(rh, lane);
                     sum_p[c] += lanes_transpose_sum(pm, lane);
                 }
@@ -248,34 +262,47 @@ mlp_residual_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
 }
 
 // ---------------------------------------------------------------- G = P^T X over the batch rows
+constexpr int kXStages = 3;                                     // ring of feature-row slices (TMA)
+constexpr uint32_t kATileBytes = kMaxHidden * 128;              // one term of P^T for a slice: up to 256 units x 64 rows, bf16
+constexpr uint32_t kXChunkBytes = kRowSlice * 128;              // 64 batch rows x 64 feature columns
+constexpr uint32_t kXStageBytes = 4 * kXChunkBytes;             // 256 feature columns
+constexpr int kBuildWarps = 8;                                  // warps 4..11 build the P^T tiles, then drain the accumulators
+
 struct GradPipe {
-    uint64_t full[kMlpStages], empty[kMlpStages];
+    uint64_t x_full[kXStages], x_empty[kXStages];
+    uint64_t a_full[2], a_empty[2];
     uint64_t acc_full, drain;
     uint32_t tmem_base;
     int abort_flag;
 };
 
+// bits (2j, 2j + 1) of `gates` -> 0xFFFF in the low / high half of the result
+__device__ __forceinline__ uint32_t pair_mask(uint32_t gates, int j) {
+    return (((gates >> (2 * j)) & 1u) ? 0x0000FFFFu : 0u) | (((gates >> (2 * j + 1)) & 1u) ? 0xFFFF0000u : 0u);
+}
+
 template <bool GATHER>
 __global__ void __launch_bounds__(kStepMlpThreads, 1)
-mlp_w1_grad_kernel(const __grid_constant__ CUtensorMap map_pt, const __grid_constant__ CUtensorMap map_x, MlpStepParams p) {
+mlp_w1_grad_kernel(const __grid_constant__ CUtensorMap map_x, MlpStepParams p) {
     extern __shared__ unsigned char smem_raw[];
-    unsigned char* ring = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    constexpr uint32_t kPtBytes = kMaxHidden * 128;                 // P^T slice: up to 256 hidden rows x 64 batch positions
-    constexpr uint32_t kXChunkBytes = kRowSlice * 128;              // 64 batch rows x 64 feature columns
-    constexpr uint32_t kStage = kPtBytes + 4 * kXChunkBytes;        // 64 KB
-    GradPipe* gp = reinterpret_cast<GradPipe*>(ring + (size_t)kMlpStages * kStage);
+    unsigned char* ring_x = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    unsigned char* ring_a = ring_x + (size_t)kXStages * kXStageBytes;           // [2 buffers][hi, lo][kATileBytes]
+    GradPipe* gp = reinterpret_cast<GradPipe*>(ring_a + 4 * (size_t)kATileBytes);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
-        for (int s = 0; s < kMlpStages; ++s) {
-            mbar_init(&gp->full[s], 1);
-            mbar_init(&gp->empty[s], 1);
+        for (int s = 0; s < kXStages; ++s) {
+            mbar_init(&gp->x_full[s], 1);
+            mbar_init(&gp->x_empty[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&gp->a_full[b], kBuildWarps);
+            mbar_init(&gp->a_empty[b], 1);
         }
         mbar_init(&gp->acc_full, 1);
         mbar_init(&gp->drain, 1);
         gp->abort_flag = 0;
         mbar_fence_init();
-        prefetch_tensormap(&map_pt);
         prefetch_tensormap(&map_x);
     }
     if (warp == 2) tmem_alloc(&gp->tmem_base, kTmemCols);
@@ -295,11 +322,13 @@ mlp_w1_grad_kernel(const __grid_constant__ CUtensorMap map_pt, const __grid_cons
     const int col0 = chunk * kFeatChunk;
     int n_q = (int)((p.d - col0 + 63) / 64);           // 64-column feature chunks that exist
     if (n_q > 4) n_q = 4;
+    const int hidden = p.g.hidden;
+    const bool two_halves = hidden > 128;
 
     if (warp == 0 || (GATHER && (warp == 3 || warp >= 12))) {
         // ------------------------------------------------------------ producer (warp 0) and, for gathered rows, seven helpers:
         // gather warp q fetches rows (q & 1) * 32 .. + 32 of 64-column chunk q >> 1 of every stage, eight four-row gathers
-        // (one per issuing lane); warp 0 also posts the expected bytes and loads the P^T box.
+        // (one per issuing lane); warp 0 also posts the expected bytes.
         const int part = warp == 0 ? 0 : (warp == 3 ? 1 : warp - 10);
         const int chunk_q = part >> 1, half = part & 1;
         int stage = 0, j = 0;
@@ -314,37 +343,35 @@ mlp_w1_grad_kernel(const __grid_constant__ CUtensorMap map_pt, const __grid_cons
                 for (int q = 0; q < 4; ++q) {
                     const int64_t i = i0 + half * 32 + lane * 4 + q;
                     long long row = i < m ? (long long)p.row_idx[i] : 0;
-                    if ((unsigned long long)row >= (unsigned long long)p.n_stored) row = 0;   // its P column is zero
+                    if ((unsigned long long)row >= (unsigned long long)p.n_stored) row = 0;   // its r is zero
                     rr[q] = (int)row;
                 }
                 r0 = rr[0]; r1 = rr[1]; r2 = rr[2]; r3 = rr[3];
             }
-            if (!mbar_wait(&gp->empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
-            unsigned char* pt_dst = ring + (size_t)stage * kStage;
-            unsigned char* x_dst = pt_dst + kPtBytes;
+            if (!mbar_wait(&gp->x_empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
+            unsigned char* x_dst = ring_x + (size_t)stage * kXStageBytes;
             if (lane == 0 && part == 0) {
-                mbar_arrive_expect_tx(&gp->full[stage], p.g.b_bytes + (uint32_t)n_q * kXChunkBytes);   // P^T box: hidden rows
-                tma_load_2d(pt_dst, &map_pt, (int)i0, 0, &gp->full[stage]);
+                mbar_arrive_expect_tx(&gp->x_full[stage], (uint32_t)n_q * kXChunkBytes);
                 if (!GATHER)
-                    for (int q = 0; q < n_q; ++q) tma_load_2d(x_dst + q * kXChunkBytes, &map_x, col0 + q * 64, (int)i0, &gp->full[stage]);
+                    for (int q = 0; q < n_q; ++q) tma_load_2d(x_dst + q * kXChunkBytes, &map_x, col0 + q * 64, (int)i0, &gp->x_full[stage]);
             }
             if (GATHER) {
                 __syncwarp();
                 if (lane < 8 && chunk_q < n_q)
                     tma_gather4(x_dst + chunk_q * kXChunkBytes + (half * 32 + lane * 4) * 128, &map_x, col0 + chunk_q * 64, r0, r1, r2, r3,
-                                &gp->full[stage]);
+                                &gp->x_full[stage]);
             }
             __syncwarp();
             ++j;
-            if (++stage == kMlpStages) { stage = 0; phase ^= 1u; }
+            if (++stage == kXStages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) {
             if (lane == 0) { latch(p.ctl, AA_ERR_SCAN_TIMEOUT); *abort_flag = 1; }
-            const int pending = j < kMlpStages ? j : kMlpStages;
+            const int pending = j < kXStages ? j : kXStages;
             for (int back = 1; back <= pending; ++back) {
-                const int jj = j - back, st = jj % kMlpStages, use = jj / kMlpStages;
+                const int jj = j - back, st = jj % kXStages, use = jj / kXStages;
                 const long long t0 = clock64();
-                while (!mbar_try_wait(&gp->full[st], (uint32_t)(use & 1)) && clock64() - t0 < kWaitCycles) {}
+                while (!mbar_try_wait(&gp->x_full[st], (uint32_t)(use & 1)) && clock64() - t0 < kWaitCycles) {}
             }
         }
     } else if (warp == 1) {
@@ -354,24 +381,31 @@ mlp_w1_grad_kernel(const __grid_constant__ CUtensorMap map_pt, const __grid_cons
         uint32_t phase = 0;
         bool ok = true;
         for (int sl = 0; sl < n_slices; ++sl) {
-            if (!mbar_wait(&gp->full[stage], phase, abort_flag)) { ok = false; break; }
+            const int buf = sl & 1;
+            if (!mbar_wait(&gp->x_full[stage], phase, abort_flag) ||
+                !mbar_wait(&gp->a_full[buf], (uint32_t)((sl >> 1) & 1), abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
             if (lane == 0) {
-                const uint32_t a_addr = smem_u32(ring + (size_t)stage * kStage);
-                const uint32_t b_addr = a_addr + kPtBytes;
+                const uint32_t b_addr = smem_u32(ring_x + (size_t)stage * kXStageBytes);
+                const uint32_t a_addr = smem_u32(ring_a + (size_t)buf * 2 * kATileBytes);
 #pragma unroll
                 for (int k = 0; k < kRowSlice / 16; ++k) {
                     // 16 batch rows = two 8-row groups (1024 bytes apart); 64-column chunks are 8192 bytes apart
                     const uint64_t b_desc = umma_smem_desc(b_addr + k * 2048, kXChunkBytes, 1024);
-                    const bool acc = (sl | k) != 0;
-                    umma_bf16(tmem_base, umma_smem_desc(a_addr + k * 32, 16, 1024), b_desc, idesc, acc);
-                    umma_bf16(tmem_base + kFeatChunk, umma_smem_desc(a_addr + 128 * 128 + k * 32, 16, 1024), b_desc, idesc, acc);
+#pragma unroll
+                    for (int term = 0; term < 2; ++term) {                      // r_hi, then r_lo, into the same accumulators
+                        const uint32_t a_term = a_addr + term * kATileBytes + k * 32;
+                        const bool acc = (sl | k | term) != 0;
+                        umma_bf16(tmem_base, umma_smem_desc(a_term, 16, 1024), b_desc, idesc, acc);
+                        if (two_halves) umma_bf16(tmem_base + kFeatChunk, umma_smem_desc(a_term + 128 * 128, 16, 1024), b_desc, idesc, acc);
+                    }
                 }
-                umma_commit(&gp->empty[stage]);
+                umma_commit(&gp->x_empty[stage]);
+                umma_commit(&gp->a_empty[buf]);
                 if (sl == n_slices - 1) umma_commit(&gp->acc_full);
             }
             __syncwarp();
-            if (++stage == kMlpStages) { stage = 0; phase ^= 1u; }
+            if (++stage == kXStages) { stage = 0; phase ^= 1u; }
         }
         if (!ok && lane == 0) { latch(p.ctl, AA_ERR_SCAN_TIMEOUT); *abort_flag = 1; }
         if (lane == 0) umma_commit(&gp->drain);
@@ -379,12 +413,57 @@ mlp_w1_grad_kernel(const __grid_constant__ CUtensorMap map_pt, const __grid_cons
         const long long t0 = clock64();
         while (!mbar_try_wait(&gp->drain, 0) && clock64() - t0 < kWaitCycles) {}
     } else if (warp >= 4 && warp < 12) {
+        // ------------------------------------------------------------ builders: P^T tiles of every slice from the gate bits and r
+        // Thread (cq, ub): the 16-byte chunk cq (batch rows 8 cq .. 8 cq + 7 of the slice) of units ub, ub + 32, ...
+        // Tile layout = what a 128-byte-swizzled TMA box [units x 64 rows] would be: unit u at u * 128 bytes, its chunk cq at
+        // position cq ^ (u & 7) within the 128-byte row.
+        const int bt = tid - 128;
+        const int cq = bt & 7, ub = bt >> 3;
+        constexpr int kUnitTrips = kMaxHidden / 32;
+        const uint32_t row_off = (uint32_t)((ub >> 3) * 1024 + (ub & 7) * 128 + ((cq ^ (ub & 7)) << 4));
+        uint32_t gates[kUnitTrips];
+        uint4 rh = make_uint4(0, 0, 0, 0), rl = make_uint4(0, 0, 0, 0);
+        auto fetch = [&](int sl) {
+            const int64_t block = s_begin + sl;
+            const uint32_t* src = p.gate_bits + block * (2 * kMaxHidden) + (cq >> 2);
+#pragma unroll
+            for (int t = 0; t < kUnitTrips; ++t) gates[t] = (ub + 32 * t) < hidden ? __ldg(src + (ub + 32 * t) * 2) : 0u;
+            rh = __ldg(reinterpret_cast<const uint4*>(p.r_hi + block * kRowSlice) + cq);
+            rl = __ldg(reinterpret_cast<const uint4*>(p.r_lo + block * kRowSlice) + cq);
+        };
+        bool ok = true;
+        if (n_slices > 0) fetch(0);
+        for (int sl = 0; sl < n_slices; ++sl) {
+            const int buf = sl & 1;
+            uint32_t g_now[kUnitTrips];
+#pragma unroll
+            for (int t = 0; t < kUnitTrips; ++t) g_now[t] = gates[t];
+            const uint4 rh_now = rh, rl_now = rl;
+            if (sl + 1 < n_slices) fetch(sl + 1);            // next slice's words are in flight while this one is built
+            if (!mbar_wait(&gp->a_empty[buf], (uint32_t)(((sl >> 1) & 1) ^ 1), abort_flag)) { ok = false; break; }
+            unsigned char* a_hi = ring_a + (size_t)buf * 2 * kATileBytes + row_off;
+#pragma unroll
+            for (int t = 0; t < kUnitTrips; ++t) {
+                if (ub + 32 * t < hidden) {
+                    const uint32_t gb = (g_now[t] >> ((cq & 3) * 8)) & 0xFFu;
+                    const uint32_t m0 = pair_mask(gb, 0), m1 = pair_mask(gb, 1), m2 = pair_mask(gb, 2), m3 = pair_mask(gb, 3);
+                    *reinterpret_cast<uint4*>(a_hi + t * 4096) = make_uint4(rh_now.x & m0, rh_now.y & m1, rh_now.z & m2, rh_now.w & m3);
+                    *reinterpret_cast<uint4*>(a_hi + kATileBytes + t * 4096) =
+                        make_uint4(rl_now.x & m0, rl_now.y & m1, rl_now.z & m2, rl_now.w & m3);
+                }
+            }
+            // the tensor cores read shared memory through the asynchronous proxy: order these plain stores before it
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&gp->a_full[buf]);
+        }
+        if (!ok && lane == 0) { latch(p.ctl, AA_ERR_SCAN_TIMEOUT); *abort_flag = 1; }
         // ------------------------------------------------------------ epilogue: this CTA's partial of G
         const int quad = warp & 3, acc = (warp - 4) >> 2;
         const int u = acc * 128 + quad * 32 + lane;                 // hidden unit
         const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kFeatChunk);
-        bool have = n_slices > 0;
-        if (have && !mbar_wait(&gp->acc_full, 0, abort_flag)) {
+        bool have = ok && n_slices > 0 && (acc == 0 || two_halves);
+        if (ok && n_slices > 0 && !mbar_wait(&gp->acc_full, 0, abort_flag)) {
             if (lane == 0) { latch(p.ctl, AA_ERR_SCAN_TIMEOUT); *abort_flag = 1; }
             have = false;
         }
@@ -514,7 +593,8 @@ __global__ void __launch_bounds__(kMaxHidden * kSmallSlices) mlp_apply_small_ker
 
 size_t mlp_step_workspace_bytes(int64_t max_rows, int64_t max_d, int64_t max_hidden, size_t* pt_bytes, size_t* small_bytes) {
     const size_t pitch = (size_t)((max_rows + kSuperRows - 1) / kSuperRows * kSuperRows);
-    *pt_bytes = ((size_t)max_hidden * pitch * 2 + 255) / 256 * 256;
+    // what the residual kernel hands to the W1-gradient kernel: gate bits (256 units per row = 32 bytes) and r as two bf16 terms
+    *pt_bytes = (pitch * (kMaxHidden / 8 + 4) + 255) / 256 * 256;
     *small_bytes = ((size_t)kMaxMlpCtas * (2 * kMaxHidden + 1) * 4 + 255) / 256 * 256;
     // split-K partials: chunks * splits <= kMaxMlpCtas CTAs, each [hidden x 256] fp32 (+ one chunk of slack per split row)
     const size_t d_pad = (size_t)((max_d + kFeatChunk - 1) / kFeatChunk * kFeatChunk);
@@ -548,8 +628,10 @@ aa_status launch_assistant_step_mlp(aa_ctx_impl* c, const MlpFeat& f, float* W1_
     p.b2 = const_cast<float*>(f.b2);
     p.d = f.d;
     p.g = make_mlp_geom(f.d, f.hidden, kHalfRows);
-    p.Pt = static_cast<__nv_bfloat16*>(c->mlp_pt);
     p.pitch = (m_host + kSuperRows - 1) / kSuperRows * kSuperRows;
+    p.gate_bits = static_cast<uint32_t*>(c->mlp_pt);
+    p.r_hi = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(c->mlp_pt) + (size_t)p.pitch * (kMaxHidden / 8));
+    p.r_lo = p.r_hi + p.pitch;
     p.small = c->mlp_small;
     p.part = c->mlp_part;
     p.d_pad = (f.d + kFeatChunk - 1) / kFeatChunk * kFeatChunk;
@@ -566,10 +648,9 @@ aa_status launch_assistant_step_mlp(aa_ctx_impl* c, const MlpFeat& f, float* W1_
     if ((size_t)splits * (size_t)f.hidden * (size_t)p.d_pad * 4 > c->mlp_part_bytes) return AA_ERR_WORKSPACE;
     p.splits = (int)splits;
 
-    alignas(64) CUtensorMap map_x, map_w, map_pt, map_xg;
+    alignas(64) CUtensorMap map_x, map_w, map_xg;
     if (!encode_bf16_tile_map(&map_x, f.x, (uint64_t)f.n, (uint64_t)f.d, (uint64_t)f.row_stride, gather ? 1 : kHalfRows) ||
         !encode_bf16_tile_map(&map_w, f.W1_bf16, (uint64_t)f.hidden, (uint64_t)f.d, (uint64_t)f.d, (uint32_t)f.hidden) ||
-        !encode_bf16_tile_map(&map_pt, p.Pt, (uint64_t)f.hidden, (uint64_t)p.pitch, (uint64_t)p.pitch, (uint32_t)f.hidden) ||
         !encode_bf16_tile_map(&map_xg, f.x, (uint64_t)f.n, (uint64_t)f.d, (uint64_t)f.row_stride, gather ? 1 : kRowSlice))
         return AA_ERR_CUDA;
 
@@ -586,10 +667,10 @@ aa_status launch_assistant_step_mlp(aa_ctx_impl* c, const MlpFeat& f, float* W1_
         if (cudaLaunchKernel(kernel, dim3(grid), dim3(kStepMlpThreads), args, smem, c->stream) != cudaSuccess) return AA_ERR_CUDA;
         ++c->launches;
         // 2. G = P^T X
-        const size_t smem2 = 1024 + (size_t)kMlpStages * (kMaxHidden * 128 + 4 * kRowSlice * 128) + sizeof(GradPipe) + 64;
+        const size_t smem2 = 1024 + (size_t)kXStages * kXStageBytes + 4 * (size_t)kATileBytes + sizeof(GradPipe) + 64;
         const void* k2 = gather ? (const void*)mlp_w1_grad_kernel<true> : (const void*)mlp_w1_grad_kernel<false>;
         if (cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2) != cudaSuccess) return AA_ERR_CUDA;
-        void* args2[] = {&map_pt, &map_xg, &p};
+        void* args2[] = {&map_xg, &p};
         if (cudaLaunchKernel(k2, dim3(p.n_chunks * p.splits), dim3(kStepMlpThreads), args2, smem2, c->stream) != cudaSuccess)
             return AA_ERR_CUDA;
         ++c->launches;

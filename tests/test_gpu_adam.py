@@ -62,8 +62,8 @@ def test_linear_dense_adam_steps(aa, n, m, d, dtype, use_rows):
         p_ref, m_ref, v_ref = O.adam(p_ref, m_ref, v_ref, np.concatenate([gw, [gb]]), LR, B1, B2, EPS, t)
         assert state.t == t
     close(np.concatenate([w.cpu().numpy(), b.cpu().numpy()]), p_ref, "params")
-    close(mom.cpu().numpy(), m_ref, "m", rel=2e-4)
-    close(var.cpu().numpy(), v_ref, "v", rel=2e-4)
+    close(mom.cpu().numpy(), m_ref, "m")
+    close(var.cpu().numpy(), v_ref, "v")
     assert np.abs(w.cpu().numpy() - p_ref[:d]).max() < 1 and np.abs(p_ref[:d]).max() > 0
 
 
@@ -93,8 +93,8 @@ def test_csr_adam_steps(aa):
         gw, gb = O.linear_grad_csr(indptr, col, val, d, s, z, row_idx=rows)
         p_ref, m_ref, v_ref = O.adam(p_ref, m_ref, v_ref, np.concatenate([gw, [gb]]), LR, B1, B2, EPS, t)
     close(np.concatenate([w.cpu().numpy(), b.cpu().numpy()]), p_ref, "params")
-    close(mom.cpu().numpy(), m_ref, "m", rel=2e-4)
-    close(var.cpu().numpy(), v_ref, "v", rel=2e-4)
+    close(mom.cpu().numpy(), m_ref, "m")
+    close(var.cpu().numpy(), v_ref, "v")
 
 
 def test_mlp_adam_steps(aa):
@@ -130,14 +130,17 @@ def test_mlp_adam_steps(aa):
         flat_p = np.concatenate([P["W1"].reshape(-1), P["b1"], P["w2"], [P["b2"]]]).astype(np.float32)
         flat_g = np.concatenate([gW1.reshape(-1), gb1, gw2, [gb2]])
         flat_p, m_ref, v_ref = O.adam(flat_p, m_ref, v_ref, flat_g, LR, B1, B2, EPS, t)
-        # What the W1 gradient may differ by: P = r [a > 0] is rounded to bf16 (2^-9 per term), and a pre-activation within
-        # 1e-4 of zero may switch its unit on or off.  Adam divides the step by sqrt(v_hat) + eps, so a gradient difference dg
-        # moves a weight by up to about lr * dg / (sqrt(v_hat) + eps) (never more than 2 lr): small gradients are amplified.
+        # What the W1 gradient may differ by: r enters the contraction as two bf16 terms (2^-17 of each row's contribution,
+        # fp32 accumulation of the same order), and the gate [a > 0] is a floating-point decision: a pre-activation within the
+        # score tolerance of zero (1e-5 of the scale of its terms) may switch its unit on or off.  Adam divides the step by
+        # sqrt(v_hat) + eps, so a gradient difference dg moves a weight by up to about lr * dg / (sqrt(v_hat) + eps) (never
+        # more than 2 lr): small gradients are amplified.
         r = np.abs(O.sigmoid(ref["s"]) - ref["z"])
-        on, near = ref["a"] > 0, np.abs(ref["a"]) < 1e-4
+        W1v = (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64).reshape(hidden, d)
+        a_scale = np.abs(P["b1"].astype(np.float64))[None, :] + np.linalg.norm(xs, axis=1)[:, None] * np.linalg.norm(W1v, axis=1)[None, :]
+        on, near = ref["a"] > 0, np.abs(ref["a"]) <= 1e-5 * a_scale
         w2a = np.abs(P["w2"].astype(np.float64))[:, None]
-        # (the bf16 roundings are independent: six standard deviations of their sum, each uniform within 2^-9 of its term)
-        dg = (6.0 * 2.0 ** -9 / math.sqrt(3.0) * np.sqrt(((r ** 2)[:, None] * on).T @ xs ** 2) + (r[:, None] * near).T @ np.abs(xs)) * w2a / m
+        dg = (2.0 ** -15 * np.sqrt(((r ** 2)[:, None] * on).T @ xs ** 2) + (r[:, None] * near).T @ np.abs(xs)) * w2a / m
         v_hat = v_ref[:hidden * d].astype(np.float64).reshape(hidden, d) / (1.0 - B2 ** t)
         slack = np.minimum(2.0 * LR, 2.0 * LR * dg / (np.sqrt(v_hat) + EPS))
         P = {"W1": flat_p[:hidden * d].reshape(hidden, d).copy(), "b1": flat_p[hidden * d:hidden * d + hidden].copy(),
@@ -146,7 +149,10 @@ def test_mlp_adam_steps(aa):
         got_W1 = W1.cpu().numpy()
         tol = 1e-4 * np.abs(P["W1"]) + 1e-4 * math.sqrt(float(np.mean(P["W1"].astype(np.float64) ** 2))) + slack
         assert np.all(np.abs(got_W1 - P["W1"]) <= tol), float(np.max(np.abs(got_W1 - P["W1"]) - tol))
-        assert float(np.mean(slack > 0.25 * LR)) < 0.05     # the amplified cases are rare: most weights are held to a small fraction of a step
+        # rounding alone is amplified past 1 % of a step for very few weights; the rest of the slack belongs to the few
+        # hidden units with a pre-activation tied at zero (each such unit touches one row of W1)
+        dg_round = 2.0 ** -15 * np.sqrt(((r ** 2)[:, None] * on).T @ xs ** 2) * w2a / m
+        assert float(np.mean(2.0 * LR * dg_round / (np.sqrt(v_hat) + EPS) > 0.01 * LR)) < 0.01 and near.mean() < 1e-3
         close(b1.cpu().numpy(), P["b1"], "b1")
         close(w2.cpu().numpy(), P["w2"], "w2")
         close([b2.item()], [P["b2"]], "b2")

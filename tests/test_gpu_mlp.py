@@ -182,6 +182,7 @@ def test_mlp_assistant_step(aa, n, m, d, hidden, use_rows, thr, lr):
     host = {k: v.cpu().numpy().copy() for k, v in (("W1", W1), ("b1", b1), ("w2", w2))}
     b2_0 = float(b2.item())
     W1b_bits = W.to_oracle(W1b).copy()
+    W1b_before = W1b.clone()
     feat = B.dense_features(x, row_idx=rows_t) if use_rows else B.dense_features(x[:m])
     cnt = torch.tensor([m], dtype=torch.int32, device=DEV)
     aa.aa_assistant_step(feat, loss, B.mlp_assistant(W1, W1b, b1, w2, b2), lr, threshold=thr, count_dev=cnt)
@@ -189,21 +190,23 @@ def test_mlp_assistant_step(aa, n, m, d, hidden, use_rows, thr, lr):
     assert aa.aa_device_status() == B.AA_OK
     ref = O.assistant_step_mlp(W.to_oracle(x), loss.cpu().numpy(), host["W1"], W1b_bits, host["b1"], host["w2"], b2_0, lr,
                                T=thr, row_idx=rows)
-    # P = r [a > 0] goes through the tensor cores in bf16 (relative rounding 2^-9 per term), and a pre-activation
-    # within 1e-4 of zero may switch its unit on or off: bound of what that does to the W1 gradient
+    # The gate [a > 0] is a decision that floating point takes: fp32 accumulation on the GPU, fp64 in the oracle.  Where the
+    # oracle's pre-activation lies within the score tolerance of zero (1e-5 of the scale of its terms) either decision is
+    # valid, and the W1 gradient may differ by that row's whole contribution; everywhere else the updated W1 is held to the
+    # plain bar.  r enters the contraction as two bf16 terms (relative error 2^-17 of each row's contribution).
     gW1 = ref["grads"][0]
     xs = (bf16_values(x) if rows is None else bf16_values(x)[rows])[:m]
     r = O.sigmoid(ref["s"]) - ref["z"]
     on = ref["a"] > 0
-    near = np.abs(ref["a"]) < 1e-4
+    W1v = bf16_values(W1b_before)
+    a_scale = np.abs(host["b1"].astype(np.float64))[None, :] + np.linalg.norm(xs, axis=1)[:, None] * np.linalg.norm(W1v, axis=1)[None, :]
+    near = np.abs(ref["a"]) <= 1e-5 * a_scale
     w2h = host["w2"].astype(np.float64)
-    bound = (np.abs(r)[:, None] * on).T @ np.abs(xs) * np.abs(w2h)[:, None] / m * 2.0 ** -8
-    bound += (np.abs(r)[:, None] * near).T @ np.abs(xs) * np.abs(w2h)[:, None] / m
-    # parameters after the update: rel 1e-4 (+ 1e-4 rms floor).  At the step sizes the workloads use (lr <= 0.1) and
-    # batches of a thousand rows or more the bf16 rounding of P is far below that bar; for a tiny batch or a step
-    # size near 1 the update itself is a large fraction of the weight and the bf16 term is allowed for explicitly.
-    plain = m >= 1000 and lr <= 0.1
-    params_close(W1.cpu().numpy(), ref["W1"], "W1", slack=None if plain else lr * bound.reshape(-1))
+    kink = (np.abs(r)[:, None] * near).T @ np.abs(xs) * np.abs(w2h)[:, None] / m
+    bound = (np.abs(r)[:, None] * on).T @ np.abs(xs) * np.abs(w2h)[:, None] / m * 2.0 ** -16 + kink
+    assert near.mean() < 1e-3                       # such ties are rare: the slack below is zero for all but a few weights
+    # parameters after the update: rel 1e-4 (+ 1e-4 rms floor), for every batch size and step size
+    params_close(W1.cpu().numpy(), ref["W1"], "W1", slack=lr * kink.reshape(-1) if near.any() else None)
     params_close(b1.cpu().numpy(), ref["b1"], "b1")
     params_close(w2.cpu().numpy(), ref["w2"], "w2")
     params_close([b2.item()], [ref["b2"]], "b2")
@@ -213,7 +216,8 @@ def test_mlp_assistant_step(aa, n, m, d, hidden, use_rows, thr, lr):
     # the gradient itself, recovered from the update (which is rounded once to fp32)
     g_gpu = (host["W1"].astype(np.float64) - W1.double().cpu().numpy()) / lr
     ulp = np.abs(host["W1"]) * 2.0 ** -23 / lr
-    assert np.all(np.abs(g_gpu - gW1) <= bound + 2 * ulp + 1e-12), float(np.max(np.abs(g_gpu - gW1) - bound - 2 * ulp))
+    fp32 = 1e-6 * (np.abs(r)[:, None] * on).T @ np.abs(xs) * np.abs(w2h)[:, None] / m     # fp32 accumulation over the batch rows
+    assert np.all(np.abs(g_gpu - gW1) <= bound + fp32 + 2 * ulp + 1e-12), float(np.max(np.abs(g_gpu - gW1) - bound - fp32 - 2 * ulp))
 
 
 def test_mlp_step_empty_batch_and_zero_lr(aa):
