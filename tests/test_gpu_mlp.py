@@ -173,6 +173,17 @@ def params_close(got, ref, what, slack=None):
     (5000, 2777, 3072, 256, True, None, 0.05), (700, 1, 128, 32, True, None, 0.1), (1300, 1300, 600, 128, False, None, 1.0),
 ])
 def test_mlp_assistant_step(aa, n, m, d, hidden, use_rows, thr, lr):
+    check_mlp_step(aa, n, m, d, hidden, use_rows, thr, lr)
+
+
+def test_mlp_assistant_step_many_tiles_per_cta_and_every_split(aa):
+    """40,000 batch rows picked out of a 65,536 x 3072 pool, hidden 256: every CTA of the forward pass runs several
+    128-row tiles through both of its alternating accumulators, and every split-K slice of the W1-gradient kernel
+    carries some fifty 64-row slices.  The whole step is checked against the oracle (about a minute of CPU time)."""
+    check_mlp_step(aa, 65536, 40000, 3072, 256, True, None, 0.01)
+
+
+def check_mlp_step(aa, n, m, d, hidden, use_rows, thr, lr):
     rng = np.random.default_rng(n + d)
     x = W.normal((n, d), 1.0, 60 + d, torch.bfloat16, DEV)
     W1, W1b, b1, w2, b2 = make_mlp(d, hidden, 61 + d)
@@ -195,7 +206,7 @@ def test_mlp_assistant_step(aa, n, m, d, hidden, use_rows, thr, lr):
     # valid, and the W1 gradient may differ by that row's whole contribution; everywhere else the updated W1 is held to the
     # plain bar.  r enters the contraction as two bf16 terms (relative error 2^-17 of each row's contribution).
     gW1 = ref["grads"][0]
-    xs = (bf16_values(x) if rows is None else bf16_values(x)[rows])[:m]
+    xs = bf16_values(x[:m] if rows is None else x[rows_t.long()])
     r = O.sigmoid(ref["s"]) - ref["z"]
     on = ref["a"] > 0
     W1v = bf16_values(W1b_before)
