@@ -2,7 +2,8 @@
 
 One step = one pass of the whole hot path over one candidate pool: Assistant score ->
 Bernoulli shrink -> ordered batch list (aa_score_shrink), per-instance Boss loss of the
-accepted batch (aa_instance_loss), labels + one Assistant SGD step (aa_assistant_step).
+accepted batch (aa_instance_loss), labels + one Assistant SGD step (aa_assistant_step_scored: the
+parameters are those the pool was screened with, so the step takes the screen's pre-activations).
 Pool: 65,536 candidates x 3072 bf16 features (403 MB, larger than L2; pools rotate),
 100-class fp32 logits, gamma 0.1, lr 0.05.  Prints ONE JSON line on rank 0.
 
@@ -551,6 +552,7 @@ def run_b200(args, cfg):
     counts = torch.zeros(n_slots, dtype=torch.int32, device=dev)
     count_of = [counts[j:j + 1] for j in range(n_slots)]
     loss = torch.zeros(cfg.n, dtype=torch.float32, device=dev)
+    score = torch.zeros(cfg.n, dtype=torch.float32, device=dev)    # pre-activations of the pool, screen -> step (same parameters)
     feats = [B.dense_features(p, id_base=base) for p, base in zip(pools, plan.id_bases)]
     batch_feats = [B.dense_features(p, row_idx=out_idx, id_base=base) for p, base in zip(pools, plan.id_bases)]
     lg = [B.logits_desc(l) for l in logits]
@@ -561,13 +563,14 @@ def run_b200(args, cfg):
         out_count = count_of[(i if slot is None else slot) % n_slots]
         if events is not None:
             events[0].record()
-        aa.aa_score_shrink(feats[k], asst, cfg.gamma, cfg.philox_seed, i, out_idx, out_count)
+        aa.aa_score_shrink(feats[k], asst, cfg.gamma, cfg.philox_seed, i, out_idx, out_count, score)
         if events is not None:
             events[1].record()
         aa.aa_instance_loss(lg[k], labels[k], loss, count_dev=out_count)
         if events is not None:
             events[2].record()
-        aa.aa_assistant_step(batch_feats[k], loss, asst, cfg.lr, count_dev=out_count)
+        # sequential schedule: the parameters are those the pool was just screened with, so the step takes the screen's scores
+        aa.aa_assistant_step_scored(batch_feats[k], loss, score, asst, cfg.lr, count_dev=out_count)
         if events is not None:
             events[3].record()
 
@@ -608,7 +611,7 @@ def run_b200(args, cfg):
     counts.zero_()
     ms_scr, best_scr, calls_scr = back_to_back(
         torch, lambda i: aa.aa_score_shrink(feats[i % npool], asst, cfg.gamma, cfg.philox_seed, 10_000 + i, out_idx,
-                                            count_of[i % n_slots]))
+                                            count_of[i % n_slots], score))
     m_scr = float(counts[3:3 + calls_scr].float().mean().item())
     if rank == 0:
         time.sleep(0.2)
@@ -645,14 +648,19 @@ def run_b200(args, cfg):
         # (weights near zero: about gamma + (1 - gamma) / 2 of the pool, the mean batch of the steps above)
         w_init, b_init = cfg.assistant(dev)
         cl = count_of[STAGE_STEPS]
-        aa.aa_score_shrink(feats[0], B.linear_assistant(w_init, b_init), cfg.gamma, cfg.philox_seed, 30_000, out_idx, cl)
+        aa.aa_score_shrink(feats[0], B.linear_assistant(w_init, b_init), cfg.gamma, cfg.philox_seed, 30_000, out_idx, cl, score)
         m_last = int(cl.item())
         ms_l, best_l, calls_l = back_to_back(torch, lambda i: aa.aa_instance_loss(lg[i % npool], labels[i % npool], loss, count_dev=cl))
-        ms_a, best_a, calls_a = back_to_back(torch, lambda i: aa.aa_assistant_step(batch_feats[i % npool], loss, asst, cfg.lr, count_dev=cl))
+        ms_a, best_a, calls_a = back_to_back(torch, lambda i: aa.aa_assistant_step_scored(batch_feats[i % npool], loss, score, asst, cfg.lr,
+                                                                                      count_dev=cl))
+        ms_r, best_r, calls_r = back_to_back(torch, lambda i: aa.aa_assistant_step(batch_feats[i % npool], loss, asst, cfg.lr, count_dev=cl))
         stages["instance_loss_alone"] = {"rows": m_last, "roofline": hbm_roofline(m_last * (cfg.classes * 4 + 8), ms_l, best_l, calls_l, peaks,
                                                                                   kernel="row_loss_short_kernel")}
-        stages["assistant_step_alone"] = {"rows": m_last, "roofline": hbm_roofline(m_last * (cfg.d * 2 + 8) + 2 * cfg.d * 4, ms_a, best_a,
-                                                                                   calls_a, peaks, kernel="linear_grad_mma_kernel")}
+        stages["assistant_step_alone"] = {"rows": m_last, "roofline": hbm_roofline(m_last * (cfg.d * 2 + 12) + 2 * cfg.d * 4, ms_a, best_a,
+                                                                                   calls_a, peaks, kernel="linear_grad_scored_kernel")}
+        stages["assistant_step_recomputing_alone"] = {
+            "rows": m_last, "what": "aa_assistant_step: the pre-activations are recomputed (any schedule)",
+            "roofline": hbm_roofline(m_last * (cfg.d * 2 + 8) + 2 * cfg.d * 4, ms_r, best_r, calls_r, peaks, kernel="linear_grad_mma_kernel")}
         assert aa.aa_device_status() == B.AA_OK
 
     # ---- the same three stages as the two-stream schedule with a Boss queue of depth k (screening runs ahead of the

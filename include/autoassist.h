@@ -277,6 +277,21 @@ aa_status aa_assistant_step(aa_ctx* ctx, const aa_feat* feat, const float* loss,
                             aa_assistant* assistant, float lr, int32_t thresh_mode, float threshold);
 
 /*
+ * Step 5 for the sequential schedule, where the parameters have not changed since the pool was screened
+ * (Algorithm 1 evaluates g(x_i; phi) for the candidates; Algorithm 2's gradient needs the same g(x_i; phi) for the
+ * batch instances as long as phi is the same): score[r] is the pre-activation s_r of STORED row r under the current
+ * parameters, as aa_score_shrink wrote it to out_score when it screened these rows without a candidate list.  The
+ * residual of batch instance i is then r_i = sigmoid(score[row_i]) - z_i and the dot products are not recomputed;
+ * everything else is aa_assistant_step.  The caller vouches that score belongs to the current parameters: after any
+ * update in between (a deeper Boss queue, a second step on one screen) use aa_assistant_step.  score = NULL is
+ * aa_assistant_step.  Kernels that have no use for the scores (CSR rows, the two-layer Assistant, rows that are not
+ * 16-byte aligned bf16 of 256..3072 features) recompute the pre-activations, so the result is the same up to rounding.
+ */
+aa_status aa_assistant_step_scored(aa_ctx* ctx, const aa_feat* feat, const float* loss, const int32_t* count_dev,
+                                   const float* score, aa_assistant* assistant, float lr, int32_t thresh_mode,
+                                   float threshold);
+
+/*
  * Step 5 with Adam in place of SGD (the paper trained its Assistants with Adam, Sec. "Image classification").  Labels and gradient exactly as
  * in aa_assistant_step; the update of every parameter p with mean gradient g is
  *   m <- beta1 m + (1 - beta1) g,   v <- beta2 v + (1 - beta2) g^2,

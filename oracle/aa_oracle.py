@@ -270,17 +270,19 @@ def screen_linear_dense(x, w, b, gamma, seed, step, id_base=0, row_idx=None):
     return {"s": s, "g": g, "p": accept_prob(g, gamma), "keep": keep, "B": compact(keep, row_idx)}
 
 
-def assistant_step_linear_dense(x, f, w, b, lr, T=None, row_idx=None):
+def assistant_step_linear_dense(x, f, w, b, lr, T=None, row_idx=None, s=None):
     """Labels from losses f, gradient under the current (w, b), one SGD update.
 
-    T=None uses the batch mean of f.  Returns (w_new fp32, b_new fp32, z).
+    T=None uses the batch mean of f.  s: optional pre-activations of the batch instances that the caller already
+    holds for these parameters (what screening computed, Algorithm 1); None evaluates them here.
+    Returns (w_new fp32, b_new fp32, z).
     """
     f = _arr(f, np.float32)
     if f.size == 0:
         return np.array(w, np.float32, copy=True), np.float32(b), np.zeros(0, np.uint8)
     T = batch_mean(f) if T is None else float(T)
     z = labels(f, T)
-    s = score_dense(x, w, b, row_idx=row_idx, n_cand=f.size)
+    s = score_dense(x, w, b, row_idx=row_idx, n_cand=f.size) if s is None else _arr(s, np.float64)
     gw, gb = linear_grad_dense(x, s, z, row_idx=row_idx)
     w_new = sgd(w, gw, lr)
     b_new = sgd(np.array([b], np.float32), np.array([gb]), lr)[0]

@@ -27,7 +27,7 @@ EXPORTS = (
     "aa_status_string", "aa_workspace_bytes", "aa_create", "aa_destroy", "aa_score_shrink",
     "aa_shrink_compact", "aa_instance_loss", "aa_assistant_step", "aa_step_host_staging_bytes", "aa_step_host",
     "aa_device_status", "aa_launch_count", "aa_shrink_compact_static", "aa_batch_cut", "aa_threshold_compact", "aa_sk_threshold", "aa_assistant_step_adam",
-    "aa_instance_loss_rows",
+    "aa_instance_loss_rows", "aa_assistant_step_scored",
 )
 AA_STATIC_MAX_CANDIDATES = 1 << 22
 
@@ -113,6 +113,8 @@ def lib() -> ctypes.CDLL:
         L.aa_instance_loss_rows.argtypes = [c_void_p, POINTER(aa_logits), c_void_p, c_void_p, c_int64, c_void_p, c_void_p]
         L.aa_assistant_step.argtypes = [c_void_p, POINTER(aa_feat), c_void_p, c_void_p, POINTER(aa_assistant),
                                         c_float, c_int32, c_float]
+        L.aa_assistant_step_scored.argtypes = [c_void_p, POINTER(aa_feat), c_void_p, c_void_p, c_void_p, POINTER(aa_assistant),
+                                               c_float, c_int32, c_float]
         L.aa_step_host_staging_bytes.argtypes = [POINTER(aa_feat), POINTER(aa_logits), POINTER(c_size_t)]
         L.aa_step_host.argtypes = [c_void_p, POINTER(aa_feat), POINTER(aa_assistant), c_float, c_uint64, c_uint64,
                                    POINTER(aa_logits), c_void_p, c_float, c_int32, c_float,
@@ -320,6 +322,16 @@ class AutoAssist:
         mode = AA_THRESH_BATCH_MEAN if threshold is None else AA_THRESH_VALUE
         self._ok(self._L.aa_assistant_step(self._ctx, byref(feat), loss.data_ptr(), _ptr(count_dev), byref(assistant),
                                            lr, mode, 0.0 if threshold is None else threshold), "aa_assistant_step")
+
+    def aa_assistant_step_scored(self, feat: aa_feat, loss: torch.Tensor, score: torch.Tensor, assistant: aa_assistant, lr: float,
+                                 threshold=None, count_dev=None):
+        """aa_assistant_step with the pre-activations that screening wrote (out_score, one per stored row): valid only
+        while the parameters are those the pool was screened with."""
+        _check(score, torch.float32, "score")
+        mode = AA_THRESH_BATCH_MEAN if threshold is None else AA_THRESH_VALUE
+        self._ok(self._L.aa_assistant_step_scored(self._ctx, byref(feat), loss.data_ptr(), _ptr(count_dev), _ptr(score),
+                                                  byref(assistant), lr, mode, 0.0 if threshold is None else threshold),
+                 "aa_assistant_step_scored")
 
     def aa_assistant_step_adam(self, feat: aa_feat, loss: torch.Tensor, assistant: aa_assistant, state: aa_adam, lr: float,
                                threshold=None, count_dev=None):

@@ -331,6 +331,15 @@ aa_status aa_assistant_step(aa_ctx* ctx, const aa_feat* feat, const float* loss,
                                      threshold);
 }
 
+aa_status aa_assistant_step_scored(aa_ctx* ctx, const aa_feat* feat, const float* loss, const int32_t* count_dev,
+                                   const float* score, aa_assistant* a, float lr, int32_t thresh_mode, float threshold) {
+    if (!ctx) return AA_ERR_INVALID_ARG;
+    ctx->impl.step_score = score;
+    const aa_status st = aa_assistant_step(ctx, feat, loss, count_dev, a, lr, thresh_mode, threshold);
+    ctx->impl.step_score = nullptr;
+    return st;
+}
+
 aa_status aa_assistant_step_adam(aa_ctx* ctx, const aa_feat* feat, const float* loss, const int32_t* count_dev, aa_assistant* a,
                                  aa_adam* state, float lr, int32_t thresh_mode, float threshold) {
     if (!ctx || !state || !state->m || !state->v || state->t < 0) return AA_ERR_INVALID_ARG;
@@ -356,7 +365,7 @@ aa_status aa_assistant_step_adam(aa_ctx* ctx, const aa_feat* feat, const float* 
 namespace {
 
 struct HostStepLayout {
-    size_t feat_off, logits_off, labels_off, idx_off, count_off, loss_off, total;
+    size_t feat_off, logits_off, labels_off, idx_off, count_off, loss_off, score_off, total;
     size_t feat_bytes, logits_bytes;
 };
 
@@ -376,6 +385,7 @@ aa_status host_step_layout(const aa_feat* feat, const aa_logits* lg, HostStepLay
     L.idx_off = off;    off = align_up(off + n * sizeof(int32_t), 256);
     L.count_off = off;  off = align_up(off + sizeof(int32_t), 256);
     L.loss_off = off;   off = align_up(off + n * sizeof(float), 256);
+    L.score_off = off;  off = align_up(off + n * sizeof(float), 256);
     L.total = off;
     return AA_OK;
 }
@@ -416,7 +426,8 @@ aa_status aa_step_host(aa_ctx* ctx, const aa_feat* feat, aa_assistant* a, float 
     }
     aa_feat f = *feat;
     f.dense = base + L.feat_off;
-    st = aa_score_shrink(ctx, &f, a, mix, seed, step, d_idx, n, d_count, nullptr, nullptr);
+    float* d_score = reinterpret_cast<float*>(base + L.score_off);
+    st = aa_score_shrink(ctx, &f, a, mix, seed, step, d_idx, n, d_count, d_score, nullptr);
     if (st != AA_OK) return st;
     aa_logits lg = *logits;
     lg.data = base + L.logits_off;
@@ -426,7 +437,8 @@ aa_status aa_step_host(aa_ctx* ctx, const aa_feat* feat, aa_assistant* a, float 
     aa_feat fb = f;
     fb.row_idx = d_idx;
     fb.n_rows = n;
-    st = aa_assistant_step(ctx, &fb, d_loss, d_count, a, lr, thresh_mode, threshold);
+    // the parameters are still those of the screening above: the step takes its pre-activations
+    st = aa_assistant_step_scored(ctx, &fb, d_loss, d_count, d_score, a, lr, thresh_mode, threshold);
     if (st != AA_OK) return st;
     // the count first, so that only the M live entries of the list and the losses cross the bus
     if (cudaMemcpyAsync(out_count, d_count, sizeof(int32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess ||

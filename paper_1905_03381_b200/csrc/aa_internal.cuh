@@ -54,6 +54,7 @@ struct aa_ctx_impl {
     float* partials;                  // gradient partial sums
     int64_t partial_floats;
     AdamArgs adam;                    // optimizer of the step being enqueued (on = 0: SGD)
+    const float* step_score;          // pre-activations handed to the step being enqueued (nullptr: recomputed)
     int64_t launches;
     uint64_t scans_since_clear;
     // two-layer Assistant step (present when the context was sized with max_hidden > 0)

@@ -315,6 +315,7 @@ aa_status launch_assistant_step_dense(aa_ctx_impl* c, const DenseFeat& f, const 
     p.m_host = m_host;
     p.count_dev = count_dev;
     p.loss = loss;
+    p.score = c->step_score;      // used by the matrix-instruction kernel; the other kernels recompute the pre-activations
     p.thresh_mode = thresh_mode;
     p.threshold = threshold;
     p.lr = lr;
@@ -326,7 +327,10 @@ aa_status launch_assistant_step_dense(aa_ctx_impl* c, const DenseFeat& f, const 
     p.d_pad = (f.d + ve - 1) / ve * ve;
     if (vec) {
         int parts = 0;
-        aa_status st = launch_assistant_grad_dense_mma(c, p, &parts);
+        aa_status st = p.score ? launch_assistant_grad_dense_scored(c, p, &parts) : AA_ERR_UNSUPPORTED;
+        if (st == AA_OK) return AA_OK;
+        if (st != AA_ERR_UNSUPPORTED) return st;
+        st = launch_assistant_grad_dense_mma(c, p, &parts);
         if (st == AA_OK) return parts > 0 ? launch_linear_apply(c, p, parts) : AA_OK;
         if (st != AA_ERR_UNSUPPORTED) return st;
         st = launch_assistant_grad_dense_tma(c, p, &parts);

@@ -17,6 +17,7 @@ struct StepParams {
     int64_t m_host;
     const int32_t* count_dev;
     const float* loss;
+    const float* score;   // optional: pre-activation of every STORED row under the current parameters (nullptr: recomputed)
     int thresh_mode;
     float threshold;
     float lr;
@@ -73,6 +74,8 @@ aa_status launch_linear_apply(aa_ctx_impl* c, const StepParams& p, int parts);
 // Matrix-instruction variant for aligned bf16 rows of 256..3072 features (a multiple of 16); AA_ERR_UNSUPPORTED otherwise.
 // *parts_out = 0 when the kernel has taken the update itself (no apply launch needed).
 aa_status launch_assistant_grad_dense_mma(aa_ctx_impl* c, StepParams& p, int* parts_out);
+// Variant for callers that pass the screening scores (p.score): same shapes as the matrix-instruction variant, no dot products.
+aa_status launch_assistant_grad_dense_scored(aa_ctx_impl* c, StepParams& p, int* parts_out);
 // Bulk-copy variant of the dense gradient kernel; AA_ERR_UNSUPPORTED when the shape does not fit its ring.
 aa_status launch_assistant_grad_dense_tma(aa_ctx_impl* c, StepParams& p, int* parts_out);
 

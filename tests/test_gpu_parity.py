@@ -421,6 +421,46 @@ def test_dense_assistant_step(aa, n, m, d, dtype, use_rows, thr):
     assert np.abs(w.cpu().numpy() - w0).max() > 0   # it did move
 
 
+@pytest.mark.parametrize("n,m,d,mix", [(4000, None, 3072, 0.3), (9000, None, 1024, 0.1), (700, None, 256, 0.5)])
+def test_dense_assistant_step_with_the_scores_of_the_screen(aa, n, m, d, mix):
+    """Sequential schedule: the step takes the pre-activations that screening wrote under the same parameters instead of
+    recomputing them.  Checked against the oracle given the same scores, against the oracle recomputing them, and
+    against the library's own recomputing route."""
+    x = W.normal((n, d), 1.0, 160 + d, torch.bfloat16, DEV)
+    w = W.normal((d,), 0.03, 161, torch.float32, DEV)
+    b = torch.full((1,), -0.2, device=DEV)
+    asst = B.linear_assistant(w, b)
+    out_idx = torch.zeros(n, dtype=torch.int32, device=DEV)
+    cnt = torch.zeros(1, dtype=torch.int32, device=DEV)
+    score = torch.zeros(n, dtype=torch.float32, device=DEV)
+    aa.aa_score_shrink(B.dense_features(x), asst, mix, 3, 7, out_idx, cnt, score)
+    torch.cuda.synchronize()
+    mm = int(cnt.item())
+    assert 0 < mm < n
+    rows = out_idx.cpu().numpy()[:mm].astype(np.int32)
+    loss = (W.normal((n,), 1.0, 162, torch.float32, DEV).abs() * 2).contiguous()
+    w0, b0 = w.cpu().numpy().copy(), float(b.item())
+    batch = B.dense_features(x, row_idx=out_idx)
+    aa.aa_assistant_step_scored(batch, loss, score, asst, 0.1, count_dev=cnt)
+    torch.cuda.synchronize()
+    w_scored, b_scored = w.cpu().numpy().copy(), float(b.item())
+    f = loss.cpu().numpy()[:mm]
+    xh = W.to_oracle(x)
+    # the oracle with the very scores the GPU used, and the oracle evaluating them itself
+    w_given, b_given, _ = O.assistant_step_linear_dense(xh, f, w0, b0, 0.1, row_idx=rows, s=score.cpu().numpy()[rows])
+    w_ref, b_ref, _ = O.assistant_step_linear_dense(xh, f, w0, b0, 0.1, row_idx=rows)
+    for wr, br in ((w_given, b_given), (w_ref, b_ref)):
+        assert_params_close(w_scored, wr)
+        assert_params_close([b_scored], [br])
+    # the recomputing route from the same starting point
+    w.copy_(torch.from_numpy(w0)); b.fill_(b0)
+    aa.aa_assistant_step(batch, loss, asst, 0.1, count_dev=cnt)
+    torch.cuda.synchronize()
+    assert_params_close(w.cpu().numpy(), w_ref)
+    assert_params_close(w.cpu().numpy(), w_scored)
+    assert np.abs(w_scored - w0).max() > 0
+
+
 def test_assistant_step_empty_batch_and_zero_lr_leave_parameters_alone(aa):
     x = W.normal((100, 32), 1.0, 1, torch.float32, DEV)
     w = W.normal((32,), 0.1, 2, torch.float32, DEV)

@@ -452,6 +452,12 @@ def test_update_special_cases():
     expect = w.copy(); expect[j] = np.float32(float(w[j]) + delta)
     assert np.array_equal(w1, expect)
     assert b1 == np.float32(0.25 + delta)
+    # handing in the pre-activation replaces the dot product and nothing else: s = 0 gives sigma = 1/2 whatever w is
+    w1s, b1s, _ = O.assistant_step_linear_dense(x, f, w, b, lr=0.5, T=1.0, s=np.array([0.0]))
+    expect_s = w.copy(); expect_s[j] = np.float32(float(w[j]) - 0.5 * (0.5 - 1.0))
+    assert np.array_equal(w1s, expect_s) and b1s == np.float32(0.25 - 0.5 * (0.5 - 1.0))
+    w1e, b1e, _ = O.assistant_step_linear_dense(x, f, w, b, lr=0.5, T=1.0, s=np.array([float(w[j]) + 0.25]))
+    assert np.array_equal(w1e, w1) and b1e == b1
     # lr = 0 and empty batch leave the parameters unchanged
     w2, b2, _ = O.assistant_step_linear_dense(x, f, w, b, lr=0.0, T=1.0)
     assert np.array_equal(w2, w) and b2 == b
