@@ -82,6 +82,27 @@ int resident_ctas(aa_ctx_impl* c, const void* kernel, int threads, size_t dyn_sm
     return ctas;
 }
 
+cudaError_t launch_overlapped(aa_ctx_impl* c, const void* kernel, dim3 grid, dim3 block, void** args, size_t smem, bool cooperative) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = c->stream;
+    cudaLaunchAttribute attrs[2];
+    unsigned int n = 0;
+    attrs[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attrs[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+    if (cooperative) {
+        attrs[n].id = cudaLaunchAttributeCooperative;
+        attrs[n].val.cooperative = 1;
+        ++n;
+    }
+    cfg.attrs = attrs;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelExC(&cfg, kernel, args);
+}
+
 namespace {
 
 bool valid_mix(float mix) { return mix >= 0.0f && mix <= 1.0f; }

@@ -100,6 +100,13 @@ __device__ __forceinline__ float adam_update(const AdamArgs& a, float param, flo
 
 __device__ __forceinline__ void latch(Control* ctl, int code) { atomicCAS(&ctl->status, 0, code); }
 
+// Programmatic dependent launch: wait for every earlier kernel of the stream to have finished (and its writes to be
+// visible); a no-op for a kernel launched in plain stream order.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel of the stream (if it was launched with programmatic serialisation) take SM resources as they
+// free up; it still waits in grid_dependency_wait() until this kernel has finished.
+__device__ __forceinline__ void grid_dependency_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -267,6 +274,13 @@ aa_status launch_assistant_step_dense(aa_ctx_impl* c, const DenseFeat& f, const 
 aa_status launch_assistant_step_csr(aa_ctx_impl* c, const CsrFeat& f, const int32_t* row_idx, int64_t n_stored,
                                     int64_t m_host, const int32_t* count_dev, const float* loss, float* w, float* b,
                                     float lr, int thresh_mode, float threshold);
+
+// Launch on the context's stream with programmatic stream serialisation: the kernel's CTAs may be placed on SMs while
+// the previous kernel of the stream is still draining (its launch latency and prologue then overlap that kernel's
+// tail).  Such a kernel MUST call grid_dependency_wait() before it reads or writes anything an earlier kernel of the
+// stream may have written; kernels that precede it call grid_dependency_release() once their own CTAs are all placed.
+// cooperative = the CTAs wait for one another (the grid must be resident at once).
+cudaError_t launch_overlapped(aa_ctx_impl* c, const void* kernel, dim3 grid, dim3 block, void** args, size_t smem, bool cooperative);
 
 // Persistent-grid size for a kernel: CTAs that fit on the device at once.
 int resident_ctas(aa_ctx_impl* c, const void* kernel, int threads, size_t dyn_smem);

@@ -122,9 +122,12 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_scored_kernel(StepPa
         cb->abort_flag = 0;
         mbar_fence_init();
     }
-    const int64_t m = batch_size(p);
     volatile int* abort_flag = &cb->abort_flag;
     __syncthreads();   // barriers are initialised
+    // everything above overlapped the previous kernel's tail; from here on its results are read (batch, losses, counters)
+    grid_dependency_wait();
+    grid_dependency_release();
+    const int64_t m = batch_size(p);
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
@@ -455,7 +458,7 @@ aa_status launch_assistant_grad_dense_scored(aa_ctx_impl* c, StepParams& p, int*
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return AA_ERR_CUDA;
     void* args[] = {&p, &g};
     // cooperative: the CTAs wait for one another before the update, so all of them must be resident at once
-    const cudaError_t le = cudaLaunchCooperativeKernel(kernel, dim3(grid), dim3(kMThreads), args, smem, c->stream);
+    const cudaError_t le = launch_overlapped(c, kernel, dim3(grid), dim3(kMThreads), args, smem, true);
     if (le == cudaErrorCooperativeLaunchTooLarge || le == cudaErrorNotSupported) {
         // the device cannot hold the whole grid at once (or has no cooperative launch): the other gradient kernels wait on nobody
         (void)cudaGetLastError();

@@ -58,6 +58,8 @@ __device__ __forceinline__ void scan_row(RunState& st, const T* row, int64_t col
 // Short rows: LPR lanes per row, several rows per warp.
 template <typename T, int LPR>
 __global__ void __launch_bounds__(256, sizeof(T) == 4 ? 6 : 4) row_loss_group_kernel(LossParams p) {
+    grid_dependency_wait();      // the row count and the logits may come from the previous kernel of the stream
+    grid_dependency_release();
     const int64_t rows = effective_rows(p);
     const int gl = threadIdx.x % LPR;
     const int64_t groups_per_grid = (int64_t)gridDim.x * (blockDim.x / LPR);
@@ -90,6 +92,8 @@ constexpr int kShortVecs = 4;
 template <typename T, int LPR>
 __global__ void __launch_bounds__(256) row_loss_short_kernel(LossParams p) {
     constexpr int VE = Vec<T>::kElems;
+    grid_dependency_wait();      // the row count and the logits may come from the previous kernel of the stream
+    grid_dependency_release();
     const int64_t rows_host = p.rows;
     int64_t rows = rows_host;
     int32_t count_raw = 0;
@@ -157,6 +161,8 @@ __global__ void __launch_bounds__(THREADS, 1536 / THREADS) row_loss_cta_kernel(L
     constexpr int kRowThreads = THREADS;
     __shared__ RunState warp_state[kRowThreads / 32];
     __shared__ unsigned int s_row[2];
+    grid_dependency_wait();      // the row count and the logits may come from the previous kernel of the stream
+    grid_dependency_release();
     const int64_t rows = effective_rows(p);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // Rows are handed out by the ticket counter (the first row of a CTA is its block index, the request for the row
@@ -265,7 +271,7 @@ aa_status launch_rows(aa_ctx_impl* c, LossParams& p) {
         grid = (int)(want < cap ? want : cap);
     }
     if (grid < 1) grid = 1;
-    if (cudaLaunchKernel(kernel, dim3(grid), dim3(threads), args, 0, c->stream) != cudaSuccess) return AA_ERR_CUDA;
+    if (launch_overlapped(c, kernel, dim3(grid), dim3(threads), args, 0, false) != cudaSuccess) return AA_ERR_CUDA;
     ++c->launches;
     return AA_OK;
 }

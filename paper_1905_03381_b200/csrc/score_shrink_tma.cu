@@ -175,10 +175,13 @@ __global__ void __launch_bounds__(kTmaThreads, 1) score_shrink_tma_kernel(DenseF
         cb->abort_flag = 0;
         mbar_fence_init();
     }
-    const float bias = *f.b;
-    const unsigned int epoch = read_epoch(p);
     volatile int* abort_flag = &cb->abort_flag;
     __syncthreads();   // barriers are initialised
+    // everything above overlapped the previous kernel's tail; from here on its results are read (weights, scan state)
+    grid_dependency_wait();
+    grid_dependency_release();
+    const float bias = *f.b;
+    const unsigned int epoch = read_epoch(p);
     // The consumer warps stage the weights among themselves (named barrier 1) while the
     // producer is already streaming rows.
     if (warp >= 1 && warp <= kConsumers) {
@@ -400,7 +403,7 @@ aa_status launch_score_shrink_dense_tma(aa_ctx_impl* c, const DenseFeat& f_in, S
     int grid = c->sm_count;
     if ((unsigned int)grid > sp.n_tiles) grid = (int)sp.n_tiles;
     void* args[] = {&f, &sp, &g};
-    if (cudaLaunchKernel(kernel, dim3(grid), dim3(kTmaThreads), args, smem, c->stream) != cudaSuccess) return AA_ERR_CUDA;
+    if (launch_overlapped(c, kernel, dim3(grid), dim3(kTmaThreads), args, smem, false) != cudaSuccess) return AA_ERR_CUDA;
     ++c->launches;
     return AA_OK;
 }
