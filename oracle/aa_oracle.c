@@ -343,6 +343,48 @@ void aa_ref_mlp_grad(const void *x, int dtype, int64_t d, int64_t row_stride,
     *grad_b2 *= inv;
 }
 
+/*
+ * Features of the convolutional Assistant (Sec. "Learning to generate smart training batches", closing
+ * paragraph: for image tasks the Assistant may be a convolution layer that shares its parameters with
+ * the Boss, followed by a pooling layer and a single linear layer).  The paper gives no sizes; the
+ * reading taken here: an instance is an image stored channel-major, x[c][y][x'] with c_in channels of
+ * height x width pixels; the convolution is the Boss's first layer, k x k taps (k odd), stride 1,
+ * zero padding (k - 1) / 2, with bias and the Boss's rectifier; the pooling layer averages
+ * non-overlapping pool x pool windows.  Output phi[c_out][height / pool][width / pool] per instance,
+ * which the single linear layer (the existing linear Assistant, the only part that trains) then scores.
+ * weight is [c_out][c_in][k][k], bias [c_out].
+ */
+void aa_ref_conv_pool_features(const void *x, int dtype, int64_t row_stride, int64_t n,
+                               int64_t c_in, int64_t height, int64_t width, int64_t c_out, int64_t k, int64_t pool,
+                               const double *weight, const double *bias, double *phi) {
+    const int64_t half = (k - 1) / 2;
+    const int64_t ph = height / pool, pw = width / pool;
+    for (int64_t i = 0; i < n; ++i) {
+        for (int64_t co = 0; co < c_out; ++co) {
+            for (int64_t py = 0; py < ph; ++py) {
+                for (int64_t px = 0; px < pw; ++px) {
+                    double window = 0.0;
+                    for (int64_t y = py * pool; y < (py + 1) * pool; ++y) {
+                        for (int64_t xx = px * pool; xx < (px + 1) * pool; ++xx) {
+                            double a = bias[co];
+                            for (int64_t ci = 0; ci < c_in; ++ci)
+                                for (int64_t dy = -half; dy <= half; ++dy)
+                                    for (int64_t dx = -half; dx <= half; ++dx) {
+                                        int64_t yy = y + dy, xs = xx + dx;
+                                        if (yy < 0 || yy >= height || xs < 0 || xs >= width) continue;   /* zero padding */
+                                        a += weight[((co * c_in + ci) * k + (dy + half)) * k + (dx + half)] *
+                                             ref_load(x, dtype, i * row_stride + (ci * height + yy) * width + xs);
+                                    }
+                            if (a > 0.0) window += a;                                                 /* rectifier */
+                        }
+                    }
+                    phi[((i * c_out + co) * ph + py) * pw + px] = window / (double)(pool * pool);     /* average pooling */
+                }
+            }
+        }
+    }
+}
+
 /* Assistant.update: plain SGD, phi <- phi - lr grad, rounded once to fp32. */
 void aa_ref_sgd(float *param, int64_t n, const double *grad, double lr) {
     for (int64_t j = 0; j < n; ++j)

@@ -244,6 +244,25 @@ def mlp_grad(x, a, s, z, w2, row_idx=None):
     return gW1, gb1, gw2, float(gb2.value)
 
 
+def conv_pool_features(x, c_in: int, height: int, width: int, weight, bias, pool: int) -> np.ndarray:
+    """Features of the convolutional Assistant: phi [n, c_out * (height // pool) * (width // pool)] in fp64.
+
+    x: [n, c_in * height * width] rows (fp32 or bf16 bits), channel-major images; weight [c_out, c_in, k, k], bias [c_out].
+    """
+    x, dt = _data(x)
+    weight = _arr(weight, np.float64)
+    bias = _arr(bias, np.float64)
+    c_out, ci, k, k2 = weight.shape
+    assert ci == c_in and k == k2 and k % 2 == 1 and height % pool == 0 and width % pool == 0
+    assert x.shape[1] == c_in * height * width
+    n = x.shape[0]
+    F = c_out * (height // pool) * (width // pool)
+    phi = np.zeros((n, F), dtype=np.float64)
+    lib().aa_ref_conv_pool_features(_p(x), dt, _c_i64(x.shape[1]), _c_i64(n), _c_i64(c_in), _c_i64(height), _c_i64(width),
+                                    _c_i64(c_out), _c_i64(k), _c_i64(pool), _p(weight), _p(bias), _p(phi))
+    return phi
+
+
 def sgd(param, grad, lr: float) -> np.ndarray:
     """Returns the updated fp32 parameters (input is not modified)."""
     out = np.array(param, dtype=np.float32, copy=True).reshape(-1)

@@ -514,6 +514,44 @@ def test_composed_csr_step_special_cases():
     assert np.array_equal(w4, w) and b4 == b
 
 
+def test_conv_pool_features_reduce_to_known_forms_and_match_torch():
+    """The convolutional Assistant's feature map (convolution with the Boss's weights, rectifier, average pooling) is
+    pinned on closed forms and on torch's float64 conv2d / avg_pool2d (library routines, not the oracle's own loops)."""
+    rng = np.random.default_rng(31)
+    n, c_in, H, Wd = 3, 3, 8, 8
+    x = rng.random((n, c_in * H * Wd)).astype(np.float32)                   # non-negative pixels
+    # identity taps (centre 1, channel c -> channel c), no bias, global average pooling: phi = per-channel mean pixel,
+    # so the linear head on phi is the linear Assistant on the pooled pixels
+    ident = np.zeros((c_in, c_in, 3, 3)); ident[np.arange(c_in), np.arange(c_in), 1, 1] = 1.0
+    phi = O.conv_pool_features(x, c_in, H, Wd, ident, np.zeros(c_in), pool=8)
+    assert phi.shape == (n, c_in)
+    assert np.allclose(phi, x.reshape(n, c_in, -1).astype(np.float64).mean(axis=2), rtol=0, atol=1e-15)
+    head = rng.normal(size=c_in)
+    assert np.allclose(phi @ head + 0.5, O.score_dense(phi.astype(np.float32), head, 0.5), atol=1e-6)
+    # zero taps: phi = relu(bias) everywhere, whatever the pooling
+    bias = np.array([0.7, -0.3, 0.0, 1.5])
+    phi0 = O.conv_pool_features(x, c_in, H, Wd, np.zeros((4, c_in, 3, 3)), bias, pool=2)
+    assert phi0.shape == (n, 4 * 4 * 4) and np.array_equal(phi0.reshape(n, 4, -1), np.broadcast_to(np.maximum(bias, 0)[None, :, None], (n, 4, 16)))
+    # a shift tap (reads the pixel to the left) shows the zero padding and the tap orientation: row y, column 0 sees 0
+    shift = np.zeros((1, 1, 3, 3)); shift[0, 0, 1, 0] = 1.0
+    img = np.arange(16, dtype=np.float32).reshape(1, 16) + 1.0
+    got = O.conv_pool_features(img, 1, 4, 4, shift, np.zeros(1), pool=1).reshape(4, 4)
+    expect = np.zeros((4, 4)); expect[:, 1:] = (img.reshape(4, 4))[:, :-1]
+    assert np.array_equal(got, expect)
+    # general case against torch in float64 (signed inputs, bias, rectifier, 2 x 2 pooling), bf16 storage widened exactly
+    xt = torch.randn((5, 3, 8, 8), dtype=torch.float32, generator=torch.Generator().manual_seed(32)).to(torch.bfloat16)
+    wt = torch.randn((6, 3, 3, 3), dtype=torch.float64, generator=torch.Generator().manual_seed(33)) * 0.4
+    bt = torch.randn((6,), dtype=torch.float64, generator=torch.Generator().manual_seed(34)) * 0.2
+    ref = torch.nn.functional.avg_pool2d(torch.relu(torch.nn.functional.conv2d(xt.double(), wt, bt, padding=1)), 2).reshape(5, -1).numpy()
+    bits = xt.reshape(5, -1).view(torch.int16).numpy().view(np.uint16)
+    mine = O.conv_pool_features(bits, 3, 8, 8, wt.numpy(), bt.numpy(), pool=2)
+    assert np.allclose(mine, ref, rtol=1e-13, atol=1e-13)
+    # 5 x 5 taps use padding 2
+    w5 = torch.randn((2, 3, 5, 5), dtype=torch.float64, generator=torch.Generator().manual_seed(35)) * 0.2
+    ref5 = torch.nn.functional.avg_pool2d(torch.relu(torch.nn.functional.conv2d(xt.double(), w5, None, padding=2)), 4).reshape(5, -1).numpy()
+    assert np.allclose(O.conv_pool_features(bits, 3, 8, 8, w5.numpy(), np.zeros(2), pool=4), ref5, rtol=1e-13, atol=1e-13)
+
+
 def test_bf16_rounding_is_nearest_even():
     src = np.array([1.0, 1.00390625, 1.01171875, -3.0e-41, 3.3895314e38, np.inf], np.float32)
     ref = torch.from_numpy(src).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
