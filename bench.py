@@ -17,6 +17,7 @@ none of them depending on --steps):
   csr                 bag-of-words screen: one 16,384-sentence pool, and 64 pools in one launch
   mlp                 two-layer Assistant shape (262,144 x 3072 bf16, hidden 256): tensor-core screen,
                       1000-class loss, two-layer step
+  conv                convolutional Assistant: feature kernel (ALU roofline) and the linear layer's screen on its features
   sweep               fused screen of 2^22 x 512 fp32, shrink+compact of 2^24 stored scores,
                       loss of 16,384 x 131,072 bf16 logits
   pipeline            the same step as the two-stream Assistant / Boss schedule
@@ -44,7 +45,7 @@ if ROOT not in sys.path:
 
 METRIC = "candidates screened/sec (score+shrink+compact -> instance loss -> Assistant step)"
 UNIT = "candidates/s"
-ALL_LEGS = ("stages", "loss", "csr", "mlp", "sweep", "pipeline", "e2e", "cpu")
+ALL_LEGS = ("stages", "loss", "csr", "mlp", "conv", "sweep", "pipeline", "e2e", "cpu")
 
 # Kernel-alone timings: REPS launches back to back between two events, LOOPS such loops, median and best loop.
 REPS = 24
@@ -456,6 +457,49 @@ def leg_mlp(torch, B, W, dev, peaks, small):
     return out
 
 
+def leg_conv(torch, B, W, dev, peaks, small, clocks_mhz):
+    """Convolutional Assistant (Boss's 3 x 3 convolution with 16 channels -> rectifier -> 4 x 4 average pooling -> linear
+    layer) on a 65,536-image pool: the feature kernel alone (plain fp32 arithmetic: an ALU roofline), then the screen of
+    the linear layer on the 1024 features per instance."""
+    cfg = W.ConvShape()
+    if small:
+        cfg.n = 8192
+    x = cfg.pool_images(0, dev)
+    weight, bias = cfg.conv(dev)
+    w, b = cfg.assistant(dev)
+    asst = B.linear_assistant(w, b)
+    F = cfg.features
+    phi = torch.zeros((cfg.n, F), dtype=torch.float32, device=dev)
+    aa = B.AutoAssist(max_rows=cfg.n, max_d=max(cfg.d, F), device=dev)
+    images, cv = B.dense_features(x), B.conv_layer(weight, bias, cfg.height, cfg.width, cfg.pool)
+    out_idx = torch.zeros(cfg.n, dtype=torch.int32, device=dev)
+    cnt = torch.zeros(1, dtype=torch.int32, device=dev)
+    ms_c, best_c, calls_c = back_to_back(torch, lambda i: aa.aa_conv_pool_features(images, cv, phi), reps=6, loops=5)
+    feat = B.dense_features(phi)
+    ms_s, best_s, calls_s = back_to_back(torch, lambda i: aa.aa_score_shrink(feat, asst, cfg.gamma, cfg.philox_seed, i, out_idx, cnt),
+                                         reps=12, loops=5)
+    assert aa.aa_device_status() == B.AA_OK
+    flops = 2.0 * cfg.n * cfg.c_out * cfg.height * cfg.width * cfg.c_in * cfg.ksize * cfg.ksize
+    sm_mhz = clocks_mhz or 1965.0
+    alu_peak = 148 * 128 * 2 * sm_mhz * 1e6 / 1e12          # fp32 lanes x 2 flop per multiply-add x SM clock
+    ach = flops / (ms_c * 1e-3) / 1e12
+    out = {
+        "workload": f"{cfg.n} images of {cfg.c_in} x {cfg.height} x {cfg.width} bf16 U[0,1), {cfg.c_out} channels of "
+                    f"{cfg.ksize} x {cfg.ksize} taps, {cfg.pool} x {cfg.pool} average pooling -> {F} fp32 features per instance",
+        "features": {"value": cfg.n / (ms_c * 1e-3), "unit": UNIT, "ms_per_call": ms_c,
+                     "roofline": {"bound": "alu", "kernel": "conv_pool_features_kernel", "achieved": ach, "peak": alu_peak,
+                                  "unit": "TFLOP/s", "frac": ach / alu_peak,
+                                  "peak_kind": f"148 SMs x 128 fp32 lanes x 2 flop x {sm_mhz:.0f} MHz (the sampled SM clock)",
+                                  "flops_per_launch": flops, "avg_launch_ms": ms_c, "best_launch_ms": best_c, "launches_timed": calls_c,
+                                  "hbm_GBs": cfg.n * (cfg.d * 2 + F * 4) / (ms_c * 1e-3) / 1e9}},
+        "linear_layer_screen": {"value": cfg.n / (ms_s * 1e-3), "unit": UNIT, "ms_per_call": ms_s, "accepted": int(cnt.item()),
+                                "roofline": hbm_roofline(cfg.n * F * 4 + F * 4 + 4 * int(cnt.item()), ms_s, best_s, calls_s, peaks,
+                                                         kernel="score_shrink_tma_kernel<float>")},
+    }
+    aa.close()
+    return out
+
+
 def leg_sweep(torch, B, W, dev, peaks, small):
     """Scaling-sweep points: fused screen of a 2^22 x 512 fp32 pool (8.6 GB), shrink+compact of 2^24 stored scores (three
     score arrays rotate: 201 MB, larger than L2), per-row loss of 16,384 x 131,072 bf16 logits (4.3 GB)."""
@@ -770,13 +814,15 @@ def run_b200(args, cfg):
     torch.cuda.empty_cache()
     mlp = leg_mlp(torch, B, W, dev, peaks, args.small) if "mlp" in legs else None
     torch.cuda.empty_cache()
+    conv = leg_conv(torch, B, W, dev, peaks, args.small, sampler.summary().get("sm_mhz")) if "conv" in legs else None
+    torch.cuda.empty_cache()
     sweep = leg_sweep(torch, B, W, dev, peaks, args.small) if "sweep" in legs else None
 
     line = {
         "metric": METRIC, "value": agg["units"] / (agg["ms"] * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": warm, "ms_per_step": agg["ms"] / K, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(cfg, args),
-        "roofline": roofline, "screen": screen, "stages": stages, "instance_loss_rows": loss_rows, "csr": csr, "mlp": mlp,
+        "roofline": roofline, "screen": screen, "stages": stages, "instance_loss_rows": loss_rows, "csr": csr, "mlp": mlp, "conv": conv,
         "sweep": sweep, "pipeline": pipeline, "cpu_baseline": cpu, "cpu_all_cores": cpu_all, "e2e": e2e,
         "gpu_launches": int(launches), "accepted_mean": accepted, "accepted_min": int(timed.min()),
         "accepted_max": int(timed.max()), "clocks": sampler.summary(),

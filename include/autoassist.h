@@ -313,6 +313,28 @@ aa_status aa_assistant_step_adam(aa_ctx* ctx, const aa_feat* feat, const float* 
                                  aa_assistant* assistant, aa_adam* state, float lr, int32_t thresh_mode, float threshold);
 
 /*
+ * Feature map of the convolutional Assistant (Sec. "Learning to generate smart training batches", closing paragraph:
+ * for image tasks the Assistant may be a convolution layer that shares its parameters with the Boss, followed by a
+ * pooling layer and a single linear layer).  The paper gives no sizes; this library's reading:
+ *   images : dense rows (fp32 or bf16), one instance per row, stored channel-major: element (ci * height + y) * width + x;
+ *            images->d = c_in * height * width; images->row_idx must be NULL (every stored row is evaluated).
+ *   conv   : the Boss's convolution: weight[c_out][c_in][ksize][ksize] and bias[c_out] (nullable) in fp32, DEVICE memory,
+ *            ksize 1, 3 or 5, stride 1, zero padding (ksize - 1) / 2, followed by the rectifier max(., 0);
+ *            pool: side of the non-overlapping average-pooling windows (divides height and width).
+ *   out_phi: row i receives phi_i[co][y / pool][x / pool] (c_out * (height / pool) * (width / pool) fp32 values),
+ *            rows phi_stride elements apart.
+ * The single linear layer is the linear Assistant on phi: screen with aa_score_shrink on a dense fp32 descriptor of
+ * out_phi, update with aa_assistant_step on the same (only that layer trains; the convolution weights stay the Boss's).
+ */
+typedef struct {
+    int32_t c_in, height, width;
+    int32_t c_out, ksize, pool;
+    const float* weight;
+    const float* bias;
+} aa_conv;
+aa_status aa_conv_pool_features(aa_ctx* ctx, const aa_feat* images, const aa_conv* conv, float* out_phi, int64_t phi_stride);
+
+/*
  * One whole step for callers whose data lives in HOST memory (pinned memory for full copy speed):
  * copies the candidate features, the Boss logits and the labels to the device staging buffer,
  * runs steps 1-5 above (dense linear Assistant), copies the batch list, its count, the

@@ -27,7 +27,7 @@ EXPORTS = (
     "aa_status_string", "aa_workspace_bytes", "aa_create", "aa_destroy", "aa_score_shrink",
     "aa_shrink_compact", "aa_instance_loss", "aa_assistant_step", "aa_step_host_staging_bytes", "aa_step_host",
     "aa_device_status", "aa_launch_count", "aa_shrink_compact_static", "aa_batch_cut", "aa_threshold_compact", "aa_sk_threshold", "aa_assistant_step_adam",
-    "aa_instance_loss_rows", "aa_assistant_step_scored",
+    "aa_instance_loss_rows", "aa_assistant_step_scored", "aa_conv_pool_features",
 )
 AA_STATIC_MAX_CANDIDATES = 1 << 22
 
@@ -54,6 +54,25 @@ class aa_logits(Structure):
         ("data", c_void_p), ("dtype", c_int32), ("reserved", c_int32),
         ("rows", c_int64), ("cols", c_int64), ("row_stride", c_int64),
     ]
+
+
+class aa_conv(Structure):
+    _fields_ = [("c_in", c_int32), ("height", c_int32), ("width", c_int32), ("c_out", c_int32), ("ksize", c_int32), ("pool", c_int32),
+                ("weight", c_void_p), ("bias", c_void_p)]
+
+
+def conv_layer(weight: torch.Tensor, bias, height: int, width: int, pool: int) -> aa_conv:
+    """The Boss's convolution for the convolutional Assistant: weight fp32 [c_out, c_in, k, k], bias fp32 [c_out] or None."""
+    _check(weight, torch.float32, "weight")
+    _check(bias, torch.float32, "bias")
+    if weight.dim() != 4 or weight.shape[2] != weight.shape[3]:
+        raise TypeError("weight must be [c_out, c_in, k, k]")
+    cv = aa_conv()
+    cv.c_out, cv.c_in, cv.ksize = weight.shape[0], weight.shape[1], weight.shape[2]
+    cv.height, cv.width, cv.pool = height, width, pool
+    cv.weight, cv.bias = weight.data_ptr(), _ptr(bias)
+    cv._keep = (weight, bias)
+    return cv
 
 
 class aa_adam(Structure):
@@ -115,6 +134,7 @@ def lib() -> ctypes.CDLL:
                                         c_float, c_int32, c_float]
         L.aa_assistant_step_scored.argtypes = [c_void_p, POINTER(aa_feat), c_void_p, c_void_p, c_void_p, POINTER(aa_assistant),
                                                c_float, c_int32, c_float]
+        L.aa_conv_pool_features.argtypes = [c_void_p, POINTER(aa_feat), POINTER(aa_conv), c_void_p, c_int64]
         L.aa_step_host_staging_bytes.argtypes = [POINTER(aa_feat), POINTER(aa_logits), POINTER(c_size_t)]
         L.aa_step_host.argtypes = [c_void_p, POINTER(aa_feat), POINTER(aa_assistant), c_float, c_uint64, c_uint64,
                                    POINTER(aa_logits), c_void_p, c_float, c_int32, c_float,
@@ -332,6 +352,15 @@ class AutoAssist:
         self._ok(self._L.aa_assistant_step_scored(self._ctx, byref(feat), loss.data_ptr(), _ptr(count_dev), _ptr(score),
                                                   byref(assistant), lr, mode, 0.0 if threshold is None else threshold),
                  "aa_assistant_step_scored")
+
+    def aa_conv_pool_features(self, images: aa_feat, conv: aa_conv, out_phi: torch.Tensor):
+        """phi = average-pooled, rectified convolution of every stored image row (the convolutional Assistant's first
+        two layers); out_phi is an fp32 [n, c_out * (height // pool) * (width // pool)] CUDA tensor with contiguous rows."""
+        if out_phi.dtype != torch.float32 or out_phi.dim() != 2 or out_phi.stride(1) != 1 or not out_phi.is_cuda:
+            raise TypeError("out_phi must be a 2-D fp32 CUDA tensor with contiguous rows")
+        self._ok(self._L.aa_conv_pool_features(self._ctx, byref(images), byref(conv), out_phi.data_ptr(),
+                                               out_phi.stride(0) if out_phi.shape[0] > 1 else out_phi.shape[1]),
+                 "aa_conv_pool_features")
 
     def aa_assistant_step_adam(self, feat: aa_feat, loss: torch.Tensor, assistant: aa_assistant, state: aa_adam, lr: float,
                                threshold=None, count_dev=None):

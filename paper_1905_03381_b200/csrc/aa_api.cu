@@ -476,6 +476,22 @@ aa_status aa_step_host(aa_ctx* ctx, const aa_feat* feat, aa_assistant* a, float 
     return AA_OK;
 }
 
+aa_status aa_conv_pool_features(aa_ctx* ctx, const aa_feat* images, const aa_conv* conv, float* out_phi, int64_t phi_stride) {
+    if (!ctx || !conv) return AA_ERR_INVALID_ARG;
+    aa_status st = check_feat(images);
+    if (st != AA_OK) return st;
+    if (images->kind != AA_FEAT_DENSE) return AA_ERR_INVALID_ARG;
+    if (images->row_idx) return AA_ERR_UNSUPPORTED;
+    if (conv->c_in <= 0 || conv->height <= 0 || conv->width <= 0 || conv->c_out <= 0 || conv->pool <= 0 || !conv->weight)
+        return AA_ERR_INVALID_ARG;
+    if (conv->ksize <= 0 || conv->ksize % 2 == 0 || conv->height % conv->pool || conv->width % conv->pool) return AA_ERR_INVALID_ARG;
+    if ((int64_t)conv->c_in * conv->height * conv->width != images->d) return AA_ERR_INVALID_ARG;
+    const int64_t feats = (int64_t)conv->c_out * (conv->height / conv->pool) * (conv->width / conv->pool);
+    if (phi_stride < feats || (images->n > 0 && !out_phi)) return AA_ERR_INVALID_ARG;
+    if (images->n == 0) return AA_OK;
+    return launch_conv_pool_features(&ctx->impl, images->dense, images->dtype, images->n, images->row_stride, *conv, out_phi, phi_stride);
+}
+
 aa_status aa_device_status(aa_ctx* ctx, int32_t* latched) {
     if (!ctx || !latched) return AA_ERR_INVALID_ARG;
     aa_ctx_impl* c = &ctx->impl;

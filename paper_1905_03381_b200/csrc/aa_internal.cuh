@@ -282,6 +282,10 @@ aa_status launch_assistant_step_csr(aa_ctx_impl* c, const CsrFeat& f, const int3
 // cooperative = the CTAs wait for one another (the grid must be resident at once).
 cudaError_t launch_overlapped(aa_ctx_impl* c, const void* kernel, dim3 grid, dim3 block, void** args, size_t smem, bool cooperative);
 
+// Convolution + rectifier + average pooling of every stored image row (the convolutional Assistant's feature map).
+aa_status launch_conv_pool_features(aa_ctx_impl* c, const void* x, int dtype, int64_t n, int64_t row_stride, const aa_conv& cv,
+                                    float* phi, int64_t phi_stride);
+
 // Persistent-grid size for a kernel: CTAs that fit on the device at once.
 int resident_ctas(aa_ctx_impl* c, const void* kernel, int threads, size_t dyn_smem);
 

@@ -185,6 +185,43 @@ class MlpShape:
 
 
 @dataclass
+class ConvShape:
+    """Convolutional Assistant case: the image shape's bf16 pixel pools read as 3 x 32 x 32 images, a first ResNet-style
+    convolution (16 channels of 3 x 3 taps ~ N(0, sqrt(2 / 27)), standing in for the Boss's) and 4 x 4 average pooling:
+    1024 features per instance for the linear layer."""
+    n: int = 65536
+    c_in: int = 3
+    height: int = 32
+    width: int = 32
+    c_out: int = 16
+    ksize: int = 3
+    pool: int = 4
+    gamma: float = 0.1
+    lr: float = 0.05
+    philox_seed: int = 0
+
+    @property
+    def d(self) -> int:
+        return self.c_in * self.height * self.width
+
+    @property
+    def features(self) -> int:
+        return self.c_out * (self.height // self.pool) * (self.width // self.pool)
+
+    def pool_images(self, pool_id: int, device="cpu") -> torch.Tensor:
+        return uniform01((self.n, self.d), 100 + pool_id, torch.bfloat16, device)
+
+    def conv(self, device="cpu"):
+        fan_in = self.c_in * self.ksize * self.ksize
+        weight = normal((self.c_out, self.c_in, self.ksize, self.ksize), float(np.sqrt(2.0 / fan_in)), 20, torch.float32, device)
+        bias = torch.zeros(self.c_out, dtype=torch.float32, device=device)
+        return weight, bias
+
+    def assistant(self, device="cpu"):
+        return linear_assistant(self.features, 21, device)
+
+
+@dataclass
 class SweepShape:
     """Scaling sweep: fp32 features ~ N(0,1), d = 512, pools of 2^20 .. 2^24 instances."""
     n: int = 1 << 20
