@@ -8,8 +8,8 @@
 //
 // The work is plain fp32 arithmetic (27 multiply-adds per output value for a 3 x 3 x 3 window, 0.44 M per 32 x 32 image
 // with 16 channels) against 6 KB of input per image: ALU-bound, not memory-bound.  One CTA holds an image (with its
-// zero border) and the taps in shared memory; a thread computes 8 adjacent outputs of two channels at a time, so that
-// every value read from shared memory feeds about five multiply-adds; the rectified outputs meet in shared memory and
+// zero border) and the taps in shared memory; a thread computes 8 adjacent outputs of four channels at a time, so that
+// every value read from shared memory feeds about four multiply-adds; the rectified outputs meet in shared memory and
 // are averaged window by window in a fixed order.
 #include "aa_internal.cuh"
 
@@ -17,8 +17,9 @@ namespace aa {
 
 namespace {
 
-constexpr int kConvThreads = 512;
+constexpr int kConvThreads = 256;
 constexpr int kSeg = 8;                 // adjacent outputs per thread and pass
+constexpr int kChan = 4;                // output channels per thread and pass
 
 struct ConvParams {
     const void* x;
@@ -30,6 +31,9 @@ struct ConvParams {
     int64_t phi_stride;
     int wp;        // padded row width in shared memory
     int hp;        // padded image height
+    int vec_rows;  // image rows can be read with 16-byte loads
+    int hpool;     // adjacent outputs a thread adds up before storing (1, 2, 4 or 8; divides pool)
+    int act_pitch; // floats per row of the rectified (partly pooled) outputs in shared memory, odd
 };
 
 template <typename T, int K>
@@ -40,40 +44,88 @@ __global__ void __launch_bounds__(kConvThreads) conv_pool_features_kernel(ConvPa
     float* w_s = conv_smem;                                  // [c_out][c_in][K][K]
     float* b_s = w_s + p.c_out * taps;                       // [c_out]
     float* img_s = b_s + ((p.c_out + 3) & ~3);               // [c_in][hp][wp], zero border
-    float* act_s = img_s + p.c_in * p.hp * p.wp;             // [c_out][height][width] rectified outputs
+    float* act_s = img_s + p.c_in * p.hp * p.wp;             // [c_out][height][act_pitch] rectified outputs, hpool of them per entry
     const int tid = threadIdx.x;
     for (int j = tid; j < p.c_out * taps; j += kConvThreads) w_s[j] = p.weight[j];
     for (int j = tid; j < p.c_out; j += kConvThreads) b_s[j] = p.bias ? p.bias[j] : 0.0f;
     for (int j = tid; j < p.c_in * p.hp * p.wp; j += kConvThreads) img_s[j] = 0.0f;
 
     const int segs = (p.width + kSeg - 1) / kSeg;
-    const int pairs = (p.c_out + 1) / 2;
-    const int items = pairs * p.height * segs;
+    const int quads = (p.c_out + kChan - 1) / kChan;
+    const int items = quads * p.height * segs;
     const int pixels = p.height * p.width;
     const int ph = p.height / p.pool, pw = p.width / p.pool;
     const int feats = p.c_out * ph * pw;
     const float inv_window = 1.0f / (float)(p.pool * p.pool);
     const T* base = static_cast<const T*>(p.x);
 
+    constexpr int VE = Vec<T>::kElems;
+    constexpr int kPre = 2;                        // vectors of the next image a thread holds while the current one is computed
+    const int n_vec = p.c_in * pixels / VE;
+    const bool prefetch = p.vec_rows && n_vec <= kPre * kConvThreads;
+    uint4 pre[kPre];
+    auto fetch = [&](int64_t img) {
+        const T* row = base + img * p.row_stride;
+#pragma unroll
+        for (int u = 0; u < kPre; ++u) {
+            const int v = tid + u * kConvThreads;
+            if (v < n_vec) pre[u] = __ldg(reinterpret_cast<const uint4*>(row) + v);
+        }
+    };
+    if (prefetch && blockIdx.x < p.n) fetch(blockIdx.x);
+
     for (int64_t img = blockIdx.x; img < p.n; img += gridDim.x) {
         __syncthreads();      // the previous image's readers are done; the first time: taps and border are in place
         const T* row = base + img * p.row_stride;
-        for (int j = tid; j < p.c_in * pixels; j += kConvThreads) {
-            const int ci = j / pixels, r = j - ci * pixels;
-            const int y = r / p.width, xx = r - y * p.width;
-            img_s[(ci * p.hp + y + H) * p.wp + xx + H] = Vec<T>::one(row + j);
+        if (prefetch) {
+            // this image's vectors were requested while the previous image was computed (a vector never straddles an
+            // image row: the width is a whole number of vectors)
+#pragma unroll
+            for (int u = 0; u < kPre; ++u) {
+                const int v = tid + u * kConvThreads;
+                if (v < n_vec) {
+                    const int j = v * VE;
+                    const int ci = j / pixels, r = j - ci * pixels;
+                    const int y = r / p.width, xx = r - y * p.width;
+                    float e[VE];
+                    Vec<T>::unpack(pre[u], e);
+                    float* dst = img_s + (ci * p.hp + y + H) * p.wp + xx + H;
+#pragma unroll
+                    for (int q = 0; q < VE; ++q) dst[q] = e[q];
+                }
+            }
+            if (img + gridDim.x < p.n) fetch(img + gridDim.x);
+        } else if (p.vec_rows) {
+            for (int v = tid; v < n_vec; v += kConvThreads) {
+                const int j = v * VE;
+                const int ci = j / pixels, r = j - ci * pixels;
+                const int y = r / p.width, xx = r - y * p.width;
+                float e[VE];
+                Vec<T>::load(row + j, e);
+                float* dst = img_s + (ci * p.hp + y + H) * p.wp + xx + H;
+#pragma unroll
+                for (int q = 0; q < VE; ++q) dst[q] = e[q];
+            }
+        } else {
+            for (int j = tid; j < p.c_in * pixels; j += kConvThreads) {
+                const int ci = j / pixels, r = j - ci * pixels;
+                const int y = r / p.width, xx = r - y * p.width;
+                img_s[(ci * p.hp + y + H) * p.wp + xx + H] = Vec<T>::one(row + j);
+            }
         }
         __syncthreads();
         for (int item = tid; item < items; item += kConvThreads) {
             const int seg = item % segs;
             const int y = (item / segs) % p.height;
-            const int cp = item / (segs * p.height);
-            const int co0 = 2 * cp, co1 = co0 + 1 < p.c_out ? co0 + 1 : co0;
-            float acc0[kSeg], acc1[kSeg];
+            const int cq = item / (segs * p.height);
+            int co[kChan];
+            float acc[kChan][kSeg];
 #pragma unroll
-            for (int q = 0; q < kSeg; ++q) { acc0[q] = b_s[co0]; acc1[q] = b_s[co1]; }
-            const float* w0 = w_s + co0 * taps;
-            const float* w1 = w_s + co1 * taps;
+            for (int c = 0; c < kChan; ++c) {
+                co[c] = cq * kChan + c < p.c_out ? cq * kChan + c : p.c_out - 1;     // a short last group repeats its last channel
+#pragma unroll
+                for (int q = 0; q < kSeg; ++q) acc[c][q] = b_s[co[c]];
+            }
             for (int ci = 0; ci < p.c_in; ++ci) {
 #pragma unroll
                 for (int dy = 0; dy < K; ++dy) {
@@ -83,21 +135,39 @@ __global__ void __launch_bounds__(kConvThreads) conv_pool_features_kernel(ConvPa
                     for (int q = 0; q < kSeg + K - 1; ++q) in[q] = in_row[q];
 #pragma unroll
                     for (int dx = 0; dx < K; ++dx) {
-                        const float t0 = w0[(ci * K + dy) * K + dx], t1 = w1[(ci * K + dy) * K + dx];
 #pragma unroll
-                        for (int q = 0; q < kSeg; ++q) {
-                            acc0[q] = fmaf(t0, in[q + dx], acc0[q]);
-                            acc1[q] = fmaf(t1, in[q + dx], acc1[q]);
+                        for (int c = 0; c < kChan; ++c) {
+                            const float t = w_s[co[c] * taps + (ci * K + dy) * K + dx];
+#pragma unroll
+                            for (int q = 0; q < kSeg; ++q) acc[c][q] = fmaf(t, in[q + dx], acc[c][q]);
                         }
                     }
                 }
             }
+            // rectifier, then the horizontal part of the pooling in registers (groups of hpool adjacent outputs, hpool = the
+            // pooling side when it divides the 8 outputs of a thread, else 1): fewer, narrower stores
 #pragma unroll
-            for (int q = 0; q < kSeg; ++q) {
-                const int xx = seg * kSeg + q;
-                if (xx < p.width) {
-                    act_s[(co0 * p.height + y) * p.width + xx] = fmaxf(acc0[q], 0.0f);
-                    if (co1 != co0) act_s[(co1 * p.height + y) * p.width + xx] = fmaxf(acc1[q], 0.0f);
+            for (int c = 0; c < kChan; ++c) {
+                if (cq * kChan + c < p.c_out) {
+                    float* dst = act_s + (co[c] * p.height + y) * p.act_pitch + (seg * kSeg) / p.hpool;
+                    if (p.hpool == 4) {
+                        const int x0 = seg * kSeg;
+                        if (x0 < p.width) dst[0] = fmaxf(acc[c][0], 0.0f) + fmaxf(acc[c][1], 0.0f) + fmaxf(acc[c][2], 0.0f) + fmaxf(acc[c][3], 0.0f);
+                        if (x0 + 4 < p.width) dst[1] = fmaxf(acc[c][4], 0.0f) + fmaxf(acc[c][5], 0.0f) + fmaxf(acc[c][6], 0.0f) + fmaxf(acc[c][7], 0.0f);
+                    } else if (p.hpool == 8) {
+                        float t = 0.0f;
+#pragma unroll
+                        for (int q = 0; q < kSeg; ++q) t += fmaxf(acc[c][q], 0.0f);
+                        if (seg * kSeg < p.width) dst[0] = t;
+                    } else if (p.hpool == 2) {
+#pragma unroll
+                        for (int q = 0; q < kSeg; q += 2)
+                            if (seg * kSeg + q < p.width) dst[q >> 1] = fmaxf(acc[c][q], 0.0f) + fmaxf(acc[c][q + 1], 0.0f);
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < kSeg; ++q)
+                            if (seg * kSeg + q < p.width) dst[q] = fmaxf(acc[c][q], 0.0f);
+                    }
                 }
             }
         }
@@ -105,10 +175,11 @@ __global__ void __launch_bounds__(kConvThreads) conv_pool_features_kernel(ConvPa
         float* out = p.phi + img * p.phi_stride;
         for (int f = tid; f < feats; f += kConvThreads) {
             const int px = f % pw, py = (f / pw) % ph, co = f / (pw * ph);
-            const float* a = act_s + (co * p.height + py * p.pool) * p.width + px * p.pool;
+            const int across = p.pool / p.hpool;          // partial sums per window row
+            const float* a = act_s + (co * p.height + py * p.pool) * p.act_pitch + px * across;
             float sum = 0.0f;
             for (int yy = 0; yy < p.pool; ++yy)
-                for (int xx = 0; xx < p.pool; ++xx) sum += a[yy * p.width + xx];
+                for (int xx = 0; xx < across; ++xx) sum += a[yy * p.act_pitch + xx];
             out[f] = sum * inv_window;
         }
     }
@@ -136,8 +207,13 @@ aa_status launch_conv_pool_features(aa_ctx_impl* c, const void* x, int dtype, in
     p.wp = segs * kSeg + cv.ksize - 1;
     if ((p.wp & 1) == 0) ++p.wp;          // odd pitch: rows of adjacent segments fall into different banks
     p.hp = cv.height + cv.ksize - 1;
+    const int es = dtype == AA_BF16 ? 2 : 4;
+    p.vec_rows = ((uintptr_t)x % 16 == 0 && (row_stride * es) % 16 == 0 && cv.width % (16 / es) == 0) ? 1 : 0;
+    p.hpool = (cv.pool == 2 || cv.pool == 4 || cv.pool == 8) ? cv.pool : ((cv.pool % 8 == 0) ? 8 : 1);
+    if (cv.width % p.hpool) p.hpool = 1;
+    p.act_pitch = ((segs * kSeg) / p.hpool) | 1;
     const size_t floats = (size_t)cv.c_out * cv.c_in * cv.ksize * cv.ksize + ((cv.c_out + 3) & ~3) + (size_t)cv.c_in * p.hp * p.wp +
-                          (size_t)cv.c_out * cv.height * cv.width;
+                          (size_t)cv.c_out * cv.height * p.act_pitch;
     const size_t smem = floats * sizeof(float);
     if (smem > 200 * 1024) return AA_ERR_UNSUPPORTED;
     const void* kernel;
