@@ -268,17 +268,25 @@ constexpr uint32_t kXChunkBytes = kRowSlice * 128;              // 64 batch rows
 constexpr uint32_t kXStageBytes = 4 * kXChunkBytes;             // 256 feature columns
 constexpr int kBuildWarps = 8;                                  // warps 4..11 build the P^T tiles, then drain the accumulators
 
+constexpr int kATiles = 4;                                      // ring of P^T tiles: r_hi and r_lo tiles of two slices
 struct GradPipe {
     uint64_t x_full[kXStages], x_empty[kXStages];
-    uint64_t a_full[2], a_empty[2];
+    uint64_t a_full[kATiles], a_empty[kATiles];
     uint64_t acc_full, drain;
     uint32_t tmem_base;
     int abort_flag;
+    uint32_t gate_lut[16];     // four gate bits (4 batch rows of one unit) -> two byte-permute selectors, see below
 };
 
-// bits (2j, 2j + 1) of `gates` -> 0xFFFF in the low / high half of the result
-__device__ __forceinline__ uint32_t pair_mask(uint32_t gates, int j) {
-    return (((gates >> (2 * j)) & 1u) ? 0x0000FFFFu : 0u) | (((gates >> (2 * j + 1)) & 1u) ? 0xFFFF0000u : 0u);
+// prmt selector that keeps (bit set) or zeroes (bit clear) each 16-bit half of a word holding two bf16 values:
+// bit 0 -> low half, bit 1 -> high half; a zeroed byte is taken from the permute's second operand (0).
+__device__ __forceinline__ uint32_t pair_selector(uint32_t two_bits) {
+    return ((two_bits & 1u) ? 0x0010u : 0x0044u) | ((two_bits & 2u) ? 0x3200u : 0x4400u);
+}
+__device__ __forceinline__ uint32_t gate_pair(uint32_t pair, uint32_t selector) {
+    uint32_t out;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(out) : "r"(pair), "r"(0u), "r"(selector));
+    return out;
 }
 
 template <bool GATHER>
@@ -286,8 +294,8 @@ __global__ void __launch_bounds__(kStepMlpThreads, 1)
 mlp_w1_grad_kernel(const __grid_constant__ CUtensorMap map_x, MlpStepParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* ring_x = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    unsigned char* ring_a = ring_x + (size_t)kXStages * kXStageBytes;           // [2 buffers][hi, lo][kATileBytes]
-    GradPipe* gp = reinterpret_cast<GradPipe*>(ring_a + 4 * (size_t)kATileBytes);
+    unsigned char* ring_a = ring_x + (size_t)kXStages * kXStageBytes;           // [kATiles][kATileBytes]: tile 2 sl + term, modulo the ring
+    GradPipe* gp = reinterpret_cast<GradPipe*>(ring_a + (size_t)kATiles * kATileBytes);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
@@ -295,7 +303,7 @@ mlp_w1_grad_kernel(const __grid_constant__ CUtensorMap map_x, MlpStepParams p) {
             mbar_init(&gp->x_full[s], 1);
             mbar_init(&gp->x_empty[s], 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < kATiles; ++b) {
             mbar_init(&gp->a_full[b], kBuildWarps);
             mbar_init(&gp->a_empty[b], 1);
         }
@@ -306,6 +314,11 @@ mlp_w1_grad_kernel(const __grid_constant__ CUtensorMap map_x, MlpStepParams p) {
         prefetch_tensormap(&map_x);
     }
     if (warp == 2) tmem_alloc(&gp->tmem_base, kTmemCols);
+    if (tid < 16) {
+        // entry b: the selectors of row pairs (0,1) and (2,3), 16 bits each
+        const uint32_t b = (uint32_t)tid;
+        gp->gate_lut[tid] = pair_selector(b & 3u) | (pair_selector((b >> 2) & 3u) << 16);
+    }
     volatile int* abort_flag = &gp->abort_flag;
     tc_fence_before_sync();
     __syncthreads();
@@ -380,31 +393,32 @@ mlp_w1_grad_kernel(const __grid_constant__ CUtensorMap map_x, MlpStepParams p) {
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
-        for (int sl = 0; sl < n_slices; ++sl) {
-            const int buf = sl & 1;
-            if (!mbar_wait(&gp->x_full[stage], phase, abort_flag) ||
-                !mbar_wait(&gp->a_full[buf], (uint32_t)((sl >> 1) & 1), abort_flag)) { ok = false; break; }
-            tc_fence_after_sync();
-            if (lane == 0) {
-                const uint32_t b_addr = smem_u32(ring_x + (size_t)stage * kXStageBytes);
-                const uint32_t a_addr = smem_u32(ring_a + (size_t)buf * 2 * kATileBytes);
+        for (int sl = 0; sl < n_slices && ok; ++sl) {
+            if (!mbar_wait(&gp->x_full[stage], phase, abort_flag)) { ok = false; break; }
+            const uint32_t b_addr = smem_u32(ring_x + (size_t)stage * kXStageBytes);
 #pragma unroll
-                for (int k = 0; k < kRowSlice / 16; ++k) {
-                    // 16 batch rows = two 8-row groups (1024 bytes apart); 64-column chunks are 8192 bytes apart
-                    const uint64_t b_desc = umma_smem_desc(b_addr + k * 2048, kXChunkBytes, 1024);
+            for (int term = 0; term < 2; ++term) {                      // r_hi, then r_lo, into the same accumulators
+                const int tile = 2 * sl + term, q = tile & (kATiles - 1);
+                if (!mbar_wait(&gp->a_full[q], (uint32_t)((tile / kATiles) & 1), abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                if (lane == 0) {
+                    const uint32_t a_addr = smem_u32(ring_a + (size_t)q * kATileBytes);
 #pragma unroll
-                    for (int term = 0; term < 2; ++term) {                      // r_hi, then r_lo, into the same accumulators
-                        const uint32_t a_term = a_addr + term * kATileBytes + k * 32;
+                    for (int k = 0; k < kRowSlice / 16; ++k) {
+                        // 16 batch rows = two 8-row groups (1024 bytes apart); 64-column chunks are 8192 bytes apart
+                        const uint64_t b_desc = umma_smem_desc(b_addr + k * 2048, kXChunkBytes, 1024);
                         const bool acc = (sl | k | term) != 0;
-                        umma_bf16(tmem_base, umma_smem_desc(a_term, 16, 1024), b_desc, idesc, acc);
-                        if (two_halves) umma_bf16(tmem_base + kFeatChunk, umma_smem_desc(a_term + 128 * 128, 16, 1024), b_desc, idesc, acc);
+                        umma_bf16(tmem_base, umma_smem_desc(a_addr + k * 32, 16, 1024), b_desc, idesc, acc);
+                        if (two_halves) umma_bf16(tmem_base + kFeatChunk, umma_smem_desc(a_addr + 128 * 128 + k * 32, 16, 1024), b_desc, idesc, acc);
+                    }
+                    umma_commit(&gp->a_empty[q]);
+                    if (term == 1) {
+                        umma_commit(&gp->x_empty[stage]);
+                        if (sl == n_slices - 1) umma_commit(&gp->acc_full);
                     }
                 }
-                umma_commit(&gp->x_empty[stage]);
-                umma_commit(&gp->a_empty[buf]);
-                if (sl == n_slices - 1) umma_commit(&gp->acc_full);
+                __syncwarp();
             }
-            __syncwarp();
             if (++stage == kXStages) { stage = 0; phase ^= 1u; }
         }
         if (!ok && lane == 0) { latch(p.ctl, AA_ERR_SCAN_TIMEOUT); *abort_flag = 1; }
@@ -433,29 +447,33 @@ mlp_w1_grad_kernel(const __grid_constant__ CUtensorMap map_x, MlpStepParams p) {
         };
         bool ok = true;
         if (n_slices > 0) fetch(0);
-        for (int sl = 0; sl < n_slices; ++sl) {
-            const int buf = sl & 1;
-            uint32_t g_now[kUnitTrips];
-#pragma unroll
-            for (int t = 0; t < kUnitTrips; ++t) g_now[t] = gates[t];
-            const uint4 rh_now = rh, rl_now = rl;
-            if (sl + 1 < n_slices) fetch(sl + 1);            // next slice's words are in flight while this one is built
-            if (!mbar_wait(&gp->a_empty[buf], (uint32_t)(((sl >> 1) & 1) ^ 1), abort_flag)) { ok = false; break; }
-            unsigned char* a_hi = ring_a + (size_t)buf * 2 * kATileBytes + row_off;
+        for (int sl = 0; sl < n_slices && ok; ++sl) {
+            // selectors of this thread's chunk for every unit it serves: one table look-up per gate byte
+            uint2 sel[kUnitTrips];
 #pragma unroll
             for (int t = 0; t < kUnitTrips; ++t) {
-                if (ub + 32 * t < hidden) {
-                    const uint32_t gb = (g_now[t] >> ((cq & 3) * 8)) & 0xFFu;
-                    const uint32_t m0 = pair_mask(gb, 0), m1 = pair_mask(gb, 1), m2 = pair_mask(gb, 2), m3 = pair_mask(gb, 3);
-                    *reinterpret_cast<uint4*>(a_hi + t * 4096) = make_uint4(rh_now.x & m0, rh_now.y & m1, rh_now.z & m2, rh_now.w & m3);
-                    *reinterpret_cast<uint4*>(a_hi + kATileBytes + t * 4096) =
-                        make_uint4(rl_now.x & m0, rl_now.y & m1, rl_now.z & m2, rl_now.w & m3);
-                }
+                const uint32_t gb = gates[t] >> ((cq & 3) * 8);
+                sel[t] = make_uint2(gp->gate_lut[gb & 0xFu], gp->gate_lut[(gb >> 4) & 0xFu]);
             }
-            // the tensor cores read shared memory through the asynchronous proxy: order these plain stores before it
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&gp->a_full[buf]);
+            const uint4 r_term[2] = {rh, rl};
+            if (sl + 1 < n_slices) fetch(sl + 1);            // next slice's words are in flight while this one is built
+#pragma unroll
+            for (int term = 0; term < 2; ++term) {
+                const int tile = 2 * sl + term, q = tile & (kATiles - 1);
+                if (!mbar_wait(&gp->a_empty[q], (uint32_t)(((tile / kATiles) & 1) ^ 1), abort_flag)) { ok = false; break; }
+                unsigned char* a_tile = ring_a + (size_t)q * kATileBytes + row_off;
+                const uint4 rv = r_term[term];
+#pragma unroll
+                for (int t = 0; t < kUnitTrips; ++t) {
+                    if (ub + 32 * t < hidden)
+                        *reinterpret_cast<uint4*>(a_tile + t * 4096) =
+                            make_uint4(gate_pair(rv.x, sel[t].x), gate_pair(rv.y, sel[t].x >> 16), gate_pair(rv.z, sel[t].y), gate_pair(rv.w, sel[t].y >> 16));
+                }
+                // the tensor cores read shared memory through the asynchronous proxy: order these plain stores before it
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&gp->a_full[q]);
+            }
         }
         if (!ok && lane == 0) { latch(p.ctl, AA_ERR_SCAN_TIMEOUT); *abort_flag = 1; }
         // ------------------------------------------------------------ epilogue: this CTA's partial of G
@@ -667,7 +685,7 @@ aa_status launch_assistant_step_mlp(aa_ctx_impl* c, const MlpFeat& f, float* W1_
         if (cudaLaunchKernel(kernel, dim3(grid), dim3(kStepMlpThreads), args, smem, c->stream) != cudaSuccess) return AA_ERR_CUDA;
         ++c->launches;
         // 2. G = P^T X
-        const size_t smem2 = 1024 + (size_t)kXStages * kXStageBytes + 4 * (size_t)kATileBytes + sizeof(GradPipe) + 64;
+        const size_t smem2 = 1024 + (size_t)kXStages * kXStageBytes + (size_t)kATiles * kATileBytes + sizeof(GradPipe) + 64;
         const void* k2 = gather ? (const void*)mlp_w1_grad_kernel<true> : (const void*)mlp_w1_grad_kernel<false>;
         if (cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2) != cudaSuccess) return AA_ERR_CUDA;
         void* args2[] = {&map_xg, &p};
