@@ -208,7 +208,10 @@ def make_csr(n, d, max_len, seed, empty_every=0):
     return indptr, col, val
 
 
-@pytest.mark.parametrize("n,d,max_len", [(1, 10, 3), (1000, 50, 6), (4099, 1 << 18, 128), (333, 1000, 700)])
+# the last three cases are large pools (many tiles per CTA): few buckets, a bucket count that is not a power of two, and the
+# translation shape's 2^18 buckets
+@pytest.mark.parametrize("n,d,max_len", [(1, 10, 3), (1000, 50, 6), (4099, 1 << 18, 128), (333, 1000, 700),
+                                         (20000, 1000, 60), (70001, 5000, 40), (131072, 1 << 18, 300)])
 def test_csr_screen(aa, n, d, max_len):
     indptr, col, val = make_csr(n, d, max_len, 50 + n, empty_every=7)
     w = W.normal((d,), 0.2, 51, torch.float32, DEV)
