@@ -1,5 +1,6 @@
 // Assistant score -> Bernoulli shrink -> ordered batch list for 16-byte aligned dense rows,
-// as one persistent, warp-specialised CTA per SM fed by bulk asynchronous copies.
+// as two persistent, warp-specialised CTAs per SM fed by bulk asynchronous copies (one CTA's start-up and tail then
+// overlap the other's streaming; together their rings hold as many bytes in flight as one CTA's ring of twice the depth).
 //
 //   producer warp : starts on tile blockIdx.x, then takes tile tickets (the next one is requested
 //                   a few stages before the current tile ends) and streams the tile's rows into a shared-memory ring with
@@ -28,11 +29,11 @@ namespace {
 
 constexpr int kMaxRowBytes = 24 * 1024;              // longest row the ring takes
 constexpr int kTargetStage = 32 * 1024;              // preferred bytes of one ring stage
-constexpr int kMaxStages = 8;
+constexpr int kMaxStages = 4;
 constexpr int kMaxSplit = 2;                         // consumer warps per stage
 constexpr int kConsumers = kMaxStages * kMaxSplit;
-constexpr int kTails = 4;                            // tail warps: tile q goes to tail q % kTails
-constexpr int kTmaThreads = (kConsumers + 1 + kTails) * 32;   // warp 0 producer, 1..16 consumers, 17..20 tails
+constexpr int kTails = 2;                            // tail warps: tile q goes to tail q % kTails
+constexpr int kTmaThreads = (kConsumers + 1 + kTails) * 32;   // warp 0 producer, 1..8 consumers, 9..10 tails
 constexpr int kSlotShift = 3;
 constexpr int kScoreSlots = 1 << kSlotShift;         // tiles in flight between consumers and tails
 constexpr int kMaxUnits = 8;                         // 32-candidate units per tile
@@ -151,7 +152,7 @@ __device__ __forceinline__ void consume_rows(const unsigned char* xs, const floa
 }
 
 template <typename T, int LPR>
-__global__ void __launch_bounds__(kTmaThreads, 1) score_shrink_tma_kernel(DenseFeat f, ShrinkParams p, TmaGeometry g) {
+__global__ void __launch_bounds__(kTmaThreads, 2) score_shrink_tma_kernel(DenseFeat f, ShrinkParams p, TmaGeometry g) {
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int VE = Vec<T>::kElems;
     unsigned char* x_ring = smem;
@@ -389,7 +390,7 @@ aa_status launch_score_shrink_dense_tma(aa_ctx_impl* c, const DenseFeat& f_in, S
 
     g.slot_rows = (tile_rows + 31) / 32 * 32;
     const size_t fixed = (size_t)g.nvec * ve * sizeof(float) + sizeof(float) * kScoreSlots * g.slot_rows + sizeof(RingControl) + 128;
-    const size_t budget = 220 * 1024;
+    const size_t budget = 110 * 1024;                  // two CTAs per SM
     if (fixed + 2 * (size_t)g.stage_bytes > budget) return AA_ERR_UNSUPPORTED;
     int stages = (int)((budget - fixed) / g.stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
@@ -400,7 +401,8 @@ aa_status launch_score_shrink_dense_tma(aa_ctx_impl* c, const DenseFeat& f_in, S
     if (st != AA_OK) return st;
     const void* kernel = f.dtype == AA_BF16 ? pick_kernel<uint16_t>(lpr) : pick_kernel<float>(lpr);
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return AA_ERR_CUDA;
-    int grid = c->sm_count;
+    int grid = resident_ctas(c, kernel, kTmaThreads, smem);     // two per SM; every CTA's first tile is its block index, so all must be resident
+    if (grid <= 0) return AA_ERR_CUDA;
     if ((unsigned int)grid > sp.n_tiles) grid = (int)sp.n_tiles;
     void* args[] = {&f, &sp, &g};
     if (launch_overlapped(c, kernel, dim3(grid), dim3(kTmaThreads), args, smem, false) != cudaSuccess) return AA_ERR_CUDA;
