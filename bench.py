@@ -406,6 +406,7 @@ def leg_mlp(torch, B, W, dev, peaks, small):
     """Two-layer Assistant shape: pool 262,144 x 3072 bf16 N(0,1), 3072 -> 256 (ReLU) -> 1, 1000-class fp32 logits,
     SGD lr 0.01 on both layers.  Screen alone (tensor roofline), loss alone, step alone on the screen's batch list, and
     whole steps."""
+    import numpy as np
     cfg = W.MlpShape()
     if small:
         cfg.n = 32768
@@ -429,11 +430,26 @@ def leg_mlp(torch, B, W, dev, peaks, small):
     ms_a, best_a, calls_a = back_to_back(torch, lambda i: aa.aa_assistant_step(batch, loss, asst, cfg.lr, count_dev=cnt),
                                          reps=10, loops=5)
 
-    def step(i):
-        aa.aa_score_shrink(feat, asst, cfg.gamma, cfg.philox_seed, 100 + i, out_idx, cnt)
-        aa.aa_instance_loss(lg, labels, loss, count_dev=cnt)
-        aa.aa_assistant_step(batch, loss, asst, cfg.lr, count_dev=cnt)
+    score = torch.zeros(cfg.n, dtype=torch.float32, device=dev)
+    marks = []
 
+    def step(i):
+        # the update takes the scores the screening wrote and the gates it left in the context's workspace
+        aa.aa_score_shrink(feat, asst, cfg.gamma, cfg.philox_seed, 100 + i, out_idx, cnt, score)
+        aa.aa_instance_loss(lg, labels, loss, count_dev=cnt)
+        if marks is not None and len(marks) < 2 * 12:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            aa.aa_assistant_step_scored(batch, loss, score, asst, cfg.lr, count_dev=cnt)
+            e1.record()
+            marks.extend((e0, e1))
+        else:
+            aa.aa_assistant_step_scored(batch, loss, score, asst, cfg.lr, count_dev=cnt)
+
+    for i in range(12):                                   # the update alone, inside whole steps (it needs a fresh screening)
+        step(i)
+    torch.cuda.synchronize()
+    ms_sc = float(np.median([marks[2 * j].elapsed_time(marks[2 * j + 1]) for j in range(len(marks) // 2)]))
     ms_w, best_w, calls_w = back_to_back(torch, step, reps=10, loops=3)
     assert aa.aa_device_status() == B.AA_OK
     flops = 2.0 * cfg.n * cfg.d * cfg.hidden
@@ -451,6 +467,9 @@ def leg_mlp(torch, B, W, dev, peaks, small):
         "assistant_step": {"ms_per_call": ms_a, "rows": m,
                            "roofline": tensor_roofline(2 * 2.0 * m * cfg.d * cfg.hidden, ms_a, best_a, calls_a, peaks,
                                                        kernel="mlp_residual_kernel + mlp_w1_grad_kernel (+ updates)")},
+        "assistant_step_scored": {"ms_per_call": ms_sc, "how": "CUDA events around the call inside 12 whole steps (median); one "
+                                  "contraction (the W1 gradient), the forward pass is the screening's",
+                                  "useful_TFLOPs": 2.0 * m * cfg.d * cfg.hidden / (ms_sc * 1e-3) / 1e12},
         "whole_step": {"value": cfg.n / (ms_w * 1e-3), "unit": UNIT, "ms_per_step": ms_w, "steps_timed": calls_w},
     }
     aa.close()

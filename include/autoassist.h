@@ -284,8 +284,16 @@ aa_status aa_assistant_step(aa_ctx* ctx, const aa_feat* feat, const float* loss,
  * residual of batch instance i is then r_i = sigmoid(score[row_i]) - z_i and the dot products are not recomputed;
  * everything else is aa_assistant_step.  The caller vouches that score belongs to the current parameters: after any
  * update in between (a deeper Boss queue, a second step on one screen) use aa_assistant_step.  score = NULL is
- * aa_assistant_step.  Kernels that have no use for the scores (CSR rows, the two-layer Assistant, rows that are not
- * 16-byte aligned bf16 of 256..3072 features) recompute the pre-activations, so the result is the same up to rounding.
+ * aa_assistant_step.  Kernels that have no use for the scores (CSR rows, rows that are not 16-byte aligned bf16 of
+ * 256..3072 features) recompute the pre-activations, so the result is the same up to rounding.
+ *
+ * Two-layer Assistant: back-propagation also needs the gates [a_iu > 0] of the hidden layer.  aa_score_shrink leaves
+ * them in this context's workspace (one bit per stored row and hidden unit) whenever it screens a dense pool without a
+ * candidate list.  The step uses score and those gates, and runs no forward pass, when the LAST two-layer screening on
+ * this context covered exactly these features (same base pointer, row count and W1_bf16 pointer), no two-layer update
+ * has gone through the context since, d is a multiple of 128 and the fp32 W1 is 16-byte aligned; grad w2 then comes
+ * from  sum_i r_i relu(a_iu) = sum_k W1b_uk G_uk + b1_u sum_i r_i [a_iu > 0]  with G the W1-gradient contraction.  In
+ * every other case the forward pass is evaluated as in aa_assistant_step and score is not read.
  */
 aa_status aa_assistant_step_scored(aa_ctx* ctx, const aa_feat* feat, const float* loss, const int32_t* count_dev,
                                    const float* score, aa_assistant* assistant, float lr, int32_t thresh_mode,

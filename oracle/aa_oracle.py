@@ -321,8 +321,11 @@ def assistant_step_linear_csr(indptr, col, val, f, w, b, lr, T=None, row_idx=Non
     return w_new, b_new, z
 
 
-def assistant_step_mlp(x, f, W1, W1_bf16, b1, w2, b2, lr, T=None, row_idx=None):
+def assistant_step_mlp(x, f, W1, W1_bf16, b1, w2, b2, lr, T=None, row_idx=None, s=None):
     """Two-layer Assistant: labels from losses f, back-propagation under the current parameters, one SGD update.
+
+    s: optional pre-activations of the batch instances that the caller already holds for these parameters (what
+    screening computed, Algorithm 1); the hidden pre-activations a are evaluated here either way.
 
     The forward pass reads the bf16 copy of W1 (uint16 bit patterns, as scoring does); the update goes to the fp32
     master, which is then rounded to nearest even into the new bf16 copy.
@@ -332,7 +335,8 @@ def assistant_step_mlp(x, f, W1, W1_bf16, b1, w2, b2, lr, T=None, row_idx=None):
     W1_vals = (np.ascontiguousarray(W1_bf16, np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
     T = batch_mean(f) if T is None else float(T)
     z = labels(f, T)
-    s, a = score_mlp(x, W1_vals, b1, w2, b2, row_idx=row_idx, n_cand=f.size, want_pre=True)
+    s_here, a = score_mlp(x, W1_vals, b1, w2, b2, row_idx=row_idx, n_cand=f.size, want_pre=True)
+    s = s_here if s is None else _arr(s, np.float64)
     gW1, gb1, gw2, gb2 = mlp_grad(x, a, s, z, w2, row_idx=row_idx)
     W1_new = sgd(W1, gW1, lr)
     return {

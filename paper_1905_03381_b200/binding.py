@@ -346,7 +346,9 @@ class AutoAssist:
     def aa_assistant_step_scored(self, feat: aa_feat, loss: torch.Tensor, score: torch.Tensor, assistant: aa_assistant, lr: float,
                                  threshold=None, count_dev=None):
         """aa_assistant_step with the pre-activations that screening wrote (out_score, one per stored row): valid only
-        while the parameters are those the pool was screened with."""
+        while the parameters are those the pool was screened with.  The two-layer Assistant also takes the gates that
+        the last screening on this context left in its workspace (same pool, same W1_bf16, no update in between);
+        otherwise it evaluates the forward pass itself."""
         _check(score, torch.float32, "score")
         mode = AA_THRESH_BATCH_MEAN if threshold is None else AA_THRESH_VALUE
         self._ok(self._L.aa_assistant_step_scored(self._ctx, byref(feat), loss.data_ptr(), _ptr(count_dev), _ptr(score),

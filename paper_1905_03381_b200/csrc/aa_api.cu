@@ -15,7 +15,7 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
     size_t tile_state_off, row_scratch_off, partials_off, total;
-    size_t mlp_pt_off, mlp_small_off, mlp_part_off, mlp_part_bytes;   // two-layer Assistant step (max_hidden > 0)
+    size_t mlp_pt_off, mlp_small_off, mlp_part_off, mlp_part_bytes, mlp_gate_off;   // two-layer Assistant step (max_hidden > 0)
     int64_t max_tiles, partial_floats;
 };
 
@@ -36,10 +36,10 @@ Layout make_layout(int64_t max_rows, int64_t max_d, int64_t max_hidden) {
     if (floats < 2 * d_pad) floats = 2 * d_pad;
     L.partial_floats = floats;
     off = align_up(off + sizeof(float) * (size_t)floats, 256);
-    L.mlp_pt_off = L.mlp_small_off = L.mlp_part_off = L.mlp_part_bytes = 0;
+    L.mlp_pt_off = L.mlp_small_off = L.mlp_part_off = L.mlp_part_bytes = L.mlp_gate_off = 0;
     if (max_hidden > 0) {
         size_t pt_bytes = 0, small_bytes = 0;
-        L.mlp_part_bytes = mlp_step_workspace_bytes(max_rows, max_d, max_hidden, &pt_bytes, &small_bytes);
+        L.mlp_part_bytes = mlp_step_workspace_bytes(max_rows, max_d, max_hidden, &pt_bytes, &small_bytes, &L.mlp_gate_off);
         L.mlp_pt_off = off;    off = align_up(off + pt_bytes, 1024);
         L.mlp_small_off = off; off = align_up(off + small_bytes, 256);
         L.mlp_part_off = off;  off = align_up(off + L.mlp_part_bytes, 256);
@@ -203,6 +203,7 @@ aa_status aa_create(aa_ctx** out, int64_t max_rows, int64_t max_d, int64_t max_h
     c.partial_floats = L.partial_floats;
     if (max_hidden > 0) {
         c.mlp_pt = c.ws + L.mlp_pt_off;
+        c.mlp_gate_cand = reinterpret_cast<uint32_t*>(c.ws + L.mlp_pt_off + L.mlp_gate_off);
         c.mlp_small = reinterpret_cast<float*>(c.ws + L.mlp_small_off);
         c.mlp_part = reinterpret_cast<float*>(c.ws + L.mlp_part_off);
         c.mlp_part_bytes = L.mlp_part_bytes;

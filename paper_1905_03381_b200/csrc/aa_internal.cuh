@@ -58,7 +58,13 @@ struct aa_ctx_impl {
     int64_t launches;
     uint64_t scans_since_clear;
     // two-layer Assistant step (present when the context was sized with max_hidden > 0)
-    void* mlp_pt;                     // bf16 [max_hidden][rows rounded up to 256]
+    void* mlp_pt;                     // gate bits and residual terms of the batch, then the gate bits of the last screened pool
+    // the gates [a > 0] that the last two-layer screening on this context left behind (32 bytes per candidate), and what
+    // they belong to: a later update on that pool's rows under unchanged parameters may use them instead of a forward pass
+    uint32_t* mlp_gate_cand;
+    const void* gate_feat;            // feature base pointer of that pool (nullptr: nothing usable)
+    const void* gate_w1;              // the bf16 first-layer weights it was screened with
+    int64_t gate_n;                   // its stored rows
     float* mlp_small;                 // per-CTA column-sum partials
     float* mlp_part;                  // split-K partials of the W1 gradient
     size_t mlp_part_bytes;
@@ -245,8 +251,10 @@ aa_status launch_score_shrink_mlp(aa_ctx_impl* c, const MlpFeat& f, ShrinkParams
 aa_status launch_assistant_step_mlp(aa_ctx_impl* c, const MlpFeat& f, float* W1_master, const int32_t* row_idx, int64_t n_stored,
                                     int64_t m_host, const int32_t* count_dev, const float* loss, float lr, int thresh_mode,
                                     float threshold);
-// Workspace of that step: returns the bytes of the split-K partials, sets the bytes of P^T and of the column-sum partials.
-size_t mlp_step_workspace_bytes(int64_t max_rows, int64_t max_d, int64_t max_hidden, size_t* pt_bytes, size_t* small_bytes);
+// Workspace of that step: returns the bytes of the split-K partials, sets the bytes of the batch hand-over + pool gate
+// bits (`pt_bytes`, the pool's gate bits start at *gate_off inside it) and of the small partials.
+size_t mlp_step_workspace_bytes(int64_t max_rows, int64_t max_d, int64_t max_hidden, size_t* pt_bytes, size_t* small_bytes,
+                                size_t* gate_off);
 
 aa_status launch_score_shrink_dense(aa_ctx_impl* c, const DenseFeat& f, ShrinkParams sp);
 // Bulk-copy (cp.async.bulk + mbarrier) variant for 16-byte aligned rows; AA_ERR_UNSUPPORTED when

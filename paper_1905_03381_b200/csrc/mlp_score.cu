@@ -42,6 +42,7 @@ struct MlpKernelParams {
     const float* w2;
     const float* b2;
     MlpGeom g;
+    uint32_t* gate_out;     // optional [candidates][kMaxHidden / 32]: bit (u & 31) of word u >> 5 = [a_u > 0] of that candidate
 };
 
 __device__ __forceinline__ void mlp_give_up(const ShrinkParams& p, TilePipe* tp) {
@@ -134,18 +135,36 @@ mlp_score_shrink_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
             }
             tc_fence_after_sync();
             float s = 0.0f;
-            for (int c0 = 0; c0 < mp.g.hidden; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld_32cols(t_row + (uint32_t)c0, r);
-                tmem_ld_wait();
+            uint32_t gate[kMaxHidden / 32];             // this candidate's gates [a_u > 0], one bit per hidden unit
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const float4 bq = reinterpret_cast<const float4*>(b1_s + c0)[q];
-                    const float4 wq = reinterpret_cast<const float4*>(w2_s + c0)[q];
-                    s = fmaf(fmaxf(__uint_as_float(r[4 * q + 0]) + bq.x, 0.0f), wq.x, s);
-                    s = fmaf(fmaxf(__uint_as_float(r[4 * q + 1]) + bq.y, 0.0f), wq.y, s);
-                    s = fmaf(fmaxf(__uint_as_float(r[4 * q + 2]) + bq.z, 0.0f), wq.z, s);
-                    s = fmaf(fmaxf(__uint_as_float(r[4 * q + 3]) + bq.w, 0.0f), wq.w, s);
+            for (int c = 0; c < kMaxHidden / 32; ++c) {
+                const int c0 = c * 32;
+                gate[c] = 0u;
+                if (c0 < mp.g.hidden) {
+                    uint32_t r[32];
+                    tmem_ld_32cols(t_row + (uint32_t)c0, r);
+                    tmem_ld_wait();
+                    // hidden is a multiple of 16: the accumulator columns past it were never written and may hold anything
+                    if (c0 + 32 > mp.g.hidden) {
+#pragma unroll
+                        for (int q = 16; q < 32; ++q) r[q] = 0u;
+                    }
+                    uint32_t bits = 0u;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const float4 bq = reinterpret_cast<const float4*>(b1_s + c0)[q];
+                        const float4 wq = reinterpret_cast<const float4*>(w2_s + c0)[q];
+                        const float a0 = __uint_as_float(r[4 * q + 0]) + bq.x, a1 = __uint_as_float(r[4 * q + 1]) + bq.y;
+                        const float a2 = __uint_as_float(r[4 * q + 2]) + bq.z, a3 = __uint_as_float(r[4 * q + 3]) + bq.w;
+                        s = fmaf(fmaxf(a0, 0.0f), wq.x, s);
+                        s = fmaf(fmaxf(a1, 0.0f), wq.y, s);
+                        s = fmaf(fmaxf(a2, 0.0f), wq.z, s);
+                        s = fmaf(fmaxf(a3, 0.0f), wq.w, s);
+                        if (!GATHER)
+                            bits |= (a0 > 0.0f ? 1u : 0u) << (4 * q) | (a1 > 0.0f ? 2u : 0u) << (4 * q) | (a2 > 0.0f ? 4u : 0u) << (4 * q) |
+                                    (a3 > 0.0f ? 8u : 0u) << (4 * q);
+                    }
+                    gate[c] = bits;
                 }
             }
             s_tile[buf * kSuperRows + row] = s + bias2;
@@ -154,6 +173,13 @@ mlp_score_shrink_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
             if (lane == 0) {
                 mbar_arrive(&tp->acc_empty[0]);
                 mbar_arrive(&cb->s_full[buf]);
+            }
+            // the gates stay behind for an update that follows this screening on the same rows (32 bytes per candidate)
+            const long long k = (long long)tile * kSuperRows + row;
+            if (!GATHER && mp.gate_out && k < p.n_cand) {
+                uint4* dst = reinterpret_cast<uint4*>(mp.gate_out + k * (kMaxHidden / 32));
+                dst[0] = make_uint4(gate[0], gate[1], gate[2], gate[3]);
+                dst[1] = make_uint4(gate[4], gate[5], gate[6], gate[7]);
             }
         }
     }
@@ -204,6 +230,12 @@ aa_status launch_score_shrink_mlp(aa_ctx_impl* c, const MlpFeat& f, ShrinkParams
     mp.g = make_mlp_geom(f.d, f.hidden);
     aa_status st = finish_shrink_params(c, sp, kSuperRows);
     if (st != AA_OK) return st;
+    // Gates of the pool's rows for a later update: only when candidate k is stored row k and the workspace has room.
+    const bool keep_gates = !gather && c->mlp_gate_cand && sp.n_cand <= c->max_rows;
+    mp.gate_out = keep_gates ? c->mlp_gate_cand : nullptr;
+    c->gate_feat = keep_gates ? f.x : nullptr;
+    c->gate_w1 = f.W1_bf16;
+    c->gate_n = sp.n_cand;
     const size_t smem = 1024 + (size_t)kMlpStages * mp.g.stage_bytes + sizeof(float) * (2 * kMaxHidden + 2 * kSuperRows) +
                         sizeof(ScoreControl) + 64;
     const void* kernel = gather ? (const void*)mlp_score_shrink_kernel<true> : (const void*)mlp_score_shrink_kernel<false>;

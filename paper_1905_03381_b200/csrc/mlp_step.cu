@@ -23,6 +23,16 @@
 //                        gradient.  Partials go to the workspace.
 //   mlp_apply_w1_kernel  W1 <- W1 - lr (w2_u / M) sum_splits G ; W1_bf16 <- round-to-nearest-even(W1).
 //   mlp_apply_small_kernel  b1, w2, b2 from the column-sum partials (reads the old w2 first).
+//
+// When the caller passes the scores of the screening that produced the batch and that screening ran on this context
+// (its gates [a > 0] are still in the workspace, one bit per candidate and unit), the forward pass is not repeated:
+//   mlp_prepare_kernel   per batch row i (stored row rho_i):  r_i = sigmoid(score[rho_i]) - z_i, its two bf16 terms, the
+//                        gate words of rho_i transposed into the block layout above, and the column sums
+//                        sum_i r_i [a_iu > 0] and sum_i r_i.
+// The W1 gradient runs as before.  grad w2 needs sum_i r_i relu(a_iu); with relu(a_iu) = [a_iu > 0] (W1b_u . x_i + b1_u) that is
+//   sum_k W1b_uk G_uk + b1_u sum_i r_i [a_iu > 0],
+// so mlp_apply_w1_kernel, which holds G and the old W1 anyway, also leaves the dot products sum_k W1b_uk G_uk (per warp,
+// added in a fixed order by mlp_apply_small_kernel).
 #include <cuda_bf16.h>
 #include <math.h>
 
@@ -65,6 +75,11 @@ struct MlpStepParams {
     float* part;              // [splits][hidden][d_pad]
     int64_t d_pad;
     int n_chunks, splits;
+    // route that reuses the screening's scores and gates (all nullptr / 0 when the forward pass is recomputed)
+    const float* score;           // pre-activation of every stored row
+    const uint32_t* gate_cand;    // [stored rows][kMaxHidden / 32] gate words of every stored row
+    float* gw2_part;              // [hidden][gw2_segs]: sum over 128 feature columns of W1b_uk G_uk
+    int gw2_segs;
     AdamArgs adam;
     Control* ctl;
 };
@@ -189,6 +204,11 @@ mlp_residual_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                 uint32_t a[32];
                 tmem_ld_32cols(t_row + (uint32_t)c0, a);
                 tmem_ld_wait();
+                // hidden is a multiple of 16: the accumulator columns past it were never written and may hold anything
+                if (c0 + 32 > hidden) {
+#pragma unroll
+                    for (int q = 16; q < 32; ++q) a[q] = 0u;
+                }
 #pragma unroll
                 for (int q = 0; q < 32; ++q) s = fmaf(fmaxf(__uint_as_float(a[q]) + b1_s[c0 + q], 0.0f), w2_s[c0 + q], s);
             }
@@ -213,6 +233,10 @@ mlp_residual_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                     uint32_t a[32];
                     tmem_ld_32cols(t_row + (uint32_t)c0, a);
                     tmem_ld_wait();
+                    if (c0 + 32 > hidden) {
+#pragma unroll
+                        for (int q = 16; q < 32; ++q) a[q] = 0u;
+                    }
                     float rh[32], pm[32];
                     uint32_t mine = 0;
 #pragma unroll
@@ -257,6 +281,115 @@ mlp_residual_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
     if (tid == 0) {
         float t = 0.0f;
         for (int w = 0; w < kStepEpiWarps; ++w) t += rsum_s[w];
+        out[2 * kMaxHidden] = t;
+    }
+}
+
+// ---------------------------------------------------------------- residuals from the screening's scores and gates
+constexpr int kPrepThreads = 1024;
+constexpr int kPrepWarps = kPrepThreads / 32;
+
+__global__ void __launch_bounds__(kPrepThreads, 1) mlp_prepare_kernel(MlpStepParams p) {
+    __shared__ double red[kPrepWarps];
+    __shared__ float col_s[kPrepWarps][kMaxHidden];      // per warp: sum_i r_i [a_iu > 0]
+    __shared__ float r_s[kPrepWarps][32];
+    __shared__ float rsum_s[kPrepWarps];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int64_t m = mlp_batch_size(p);
+    // shrinking threshold T: the caller's value or the batch mean; every CTA adds the losses in the same order
+    double T_shrink = (double)p.threshold;
+    if (p.thresh_mode != AA_THRESH_VALUE) {
+        double acc = 0.0;
+        if (((uintptr_t)p.loss & 15) == 0) {
+            const int64_t quads = m >> 2;
+            for (int64_t q = tid; q < quads; q += kPrepThreads) {
+                const float4 v = __ldg(reinterpret_cast<const float4*>(p.loss) + q);
+                acc += ((double)v.x + (double)v.y) + ((double)v.z + (double)v.w);
+            }
+            for (int64_t i = (quads << 2) + tid; i < m; i += kPrepThreads) acc += (double)__ldg(p.loss + i);
+        } else {
+            for (int64_t i = tid; i < m; i += kPrepThreads) acc += (double)__ldg(p.loss + i);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+        if (lane == 0) red[warp] = acc;
+        __syncthreads();
+        double total = 0.0;
+        for (int wi = 0; wi < kPrepWarps; ++wi) total += red[wi];
+        T_shrink = m > 0 ? total / (double)m : 0.0;
+    }
+    float sum_p[kMaxHidden / 32];                        // lane l: units c * 32 + l over this warp's rows
+#pragma unroll
+    for (int c = 0; c < kMaxHidden / 32; ++c) sum_p[c] = 0.0f;
+    float sum_r = 0.0f;
+    // groups of 32 adjacent batch rows, up to the end of the last 64-row slice the W1-gradient kernel reads
+    const int64_t n_groups = ((m + kRowSlice - 1) / kRowSlice) * (kRowSlice / 32);
+    for (int64_t g = (int64_t)blockIdx.x * kPrepWarps + warp; g < n_groups; g += (int64_t)gridDim.x * kPrepWarps) {
+        const int64_t i = g * 32 + lane;
+        bool valid = i < m;
+        long long row = 0;
+        if (valid) {
+            row = p.row_idx ? (long long)p.row_idx[i] : (long long)i;
+            if ((unsigned long long)row >= (unsigned long long)p.n_stored) {
+                latch(p.ctl, AA_ERR_BAD_INDEX);
+                valid = false;
+            }
+        }
+        float r = 0.0f;
+        uint4 g_lo = make_uint4(0, 0, 0, 0), g_hi = make_uint4(0, 0, 0, 0);
+        if (valid) {
+            const float f_i = __ldg(p.loss + i);
+            const float z = (double)f_i > T_shrink ? 1.0f : 0.0f;
+            r = sigmoid_f32(__ldg(p.score + row)) - z;
+            const uint4* src = reinterpret_cast<const uint4*>(p.gate_cand + row * (kMaxHidden / 32));
+            g_lo = __ldg(src);
+            g_hi = __ldg(src + 1);
+        }
+        sum_r += r;
+        {
+            const __nv_bfloat16 hi = __float2bfloat16_rn(r);
+            p.r_hi[i] = hi;
+            p.r_lo[i] = __float2bfloat16_rn(r - __bfloat162float(hi));
+        }
+        __syncwarp();
+        r_s[warp][lane] = r;
+        __syncwarp();
+        const uint32_t words[kMaxHidden / 32] = {g_lo.x, g_lo.y, g_lo.z, g_lo.w, g_hi.x, g_hi.y, g_hi.z, g_hi.w};
+        uint32_t* gate_dst = p.gate_bits + (g >> 1) * (2 * kMaxHidden) + (g & 1);
+#pragma unroll
+        for (int c = 0; c < kMaxHidden / 32; ++c) {
+            if (c * 32 < p.g.hidden) {
+                // 32 x 32 bit transpose: lane q ends with unit c * 32 + q over the warp's rows
+                uint32_t mine = 0;
+#pragma unroll
+                for (int q = 0; q < 32; ++q) {
+                    const uint32_t rows_of_unit = __ballot_sync(0xFFFFFFFFu, (words[c] >> q) & 1u);
+                    if (lane == q) mine = rows_of_unit;
+                }
+                gate_dst[(c * 32 + lane) * 2] = mine;
+                float acc = 0.0f;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) acc += ((mine >> j) & 1u) ? r_s[warp][j] : 0.0f;
+                sum_p[c] += acc;
+            }
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < kMaxHidden / 32; ++c) col_s[warp][c * 32 + lane] = sum_p[c];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum_r += __shfl_xor_sync(0xFFFFFFFFu, sum_r, o);
+    if (lane == 0) rsum_s[warp] = sum_r;
+    __syncthreads();
+    float* out = p.small + (int64_t)blockIdx.x * (2 * kMaxHidden + 1);
+    if (tid < kMaxHidden) {
+        float t = 0.0f;
+        for (int w = 0; w < kPrepWarps; ++w) t += col_s[w][tid];
+        out[tid] = 0.0f;                                  // grad w2 comes from the W1-gradient partials on this route
+        out[kMaxHidden + tid] = t;
+    }
+    if (tid == 0) {
+        float t = 0.0f;
+        for (int w = 0; w < kPrepWarps; ++w) t += rsum_s[w];
         out[2 * kMaxHidden] = t;
     }
 }
@@ -531,6 +664,18 @@ __global__ void __launch_bounds__(256) mlp_apply_w1_kernel(MlpStepParams p) {
             float4* wp = reinterpret_cast<float4*>(p.W1 + u * p.d + k);
             float4 w = *wp;
             const float gv[4] = {g.x, g.y, g.z, g.w};
+            if (p.gw2_part) {
+                // sum_k W1b_uk G_uk over this warp's 128 columns of unit u (d is a multiple of 128 on this route, so the
+                // 32 lanes share u), with the bf16 weights the screening multiplied with
+                const uint2 wb = *reinterpret_cast<const uint2*>(p.W1_bf16 + u * p.d + k);
+                float dot = __uint_as_float(wb.x << 16) * g.x;
+                dot = fmaf(__uint_as_float(wb.x & 0xFFFF0000u), g.y, dot);
+                dot = fmaf(__uint_as_float(wb.y << 16), g.z, dot);
+                dot = fmaf(__uint_as_float(wb.y & 0xFFFF0000u), g.w, dot);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, o);
+                if ((threadIdx.x & 31) == 0) p.gw2_part[u * p.gw2_segs + (k >> 7)] = dot;
+            }
             float wv[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e)
@@ -589,6 +734,12 @@ __global__ void __launch_bounds__(kMaxHidden * kSmallSlices) mlp_apply_small_ker
             g_w2 += part_w2[q][u];
             g_b1 += part_b1[q][u];
         }
+        if (p.gw2_part) {
+            // sum_i r_i relu(a_iu) = sum_k W1b_uk G_uk + b1_u sum_i r_i [a_iu > 0]  (b1 still holds the old value)
+            float t = 0.0f;
+            for (int seg = 0; seg < p.gw2_segs; ++seg) t += p.gw2_part[u * p.gw2_segs + seg];
+            g_w2 = fmaf(p.b1[u], g_b1, t);
+        }
         const float w2_old = p.w2[u];
         const int64_t hd = (int64_t)p.g.hidden * p.d;      // moments: W1, then b1, w2, b2
         if (p.adam.on) {
@@ -609,11 +760,17 @@ __global__ void __launch_bounds__(kMaxHidden * kSmallSlices) mlp_apply_small_ker
 
 }  // namespace
 
-size_t mlp_step_workspace_bytes(int64_t max_rows, int64_t max_d, int64_t max_hidden, size_t* pt_bytes, size_t* small_bytes) {
+constexpr size_t kSmallBytes = ((size_t)kMaxMlpCtas * (2 * kMaxHidden + 1) * 4 + 255) / 256 * 256;
+
+size_t mlp_step_workspace_bytes(int64_t max_rows, int64_t max_d, int64_t max_hidden, size_t* pt_bytes, size_t* small_bytes,
+                                size_t* gate_off) {
     const size_t pitch = (size_t)((max_rows + kSuperRows - 1) / kSuperRows * kSuperRows);
-    // what the residual kernel hands to the W1-gradient kernel: gate bits (256 units per row = 32 bytes) and r as two bf16 terms
-    *pt_bytes = (pitch * (kMaxHidden / 8 + 4) + 255) / 256 * 256;
-    *small_bytes = ((size_t)kMaxMlpCtas * (2 * kMaxHidden + 1) * 4 + 255) / 256 * 256;
+    // what the residual kernel hands to the W1-gradient kernel: gate bits (256 units per row = 32 bytes) and r as two bf16
+    // terms; behind it the gate words the last screening left for every row of its pool (32 bytes per row)
+    *gate_off = (pitch * (kMaxHidden / 8 + 4) + 255) / 256 * 256;
+    *pt_bytes = *gate_off + (pitch * (kMaxHidden / 8) + 255) / 256 * 256;
+    // per-CTA column sums, then the per-warp dot products of the grad-w2 identity ([kMaxHidden][max_d / 128])
+    *small_bytes = kSmallBytes + ((size_t)kMaxHidden * (size_t)((max_d + 127) / 128) * 4 + 255) / 256 * 256;
     // split-K partials: chunks * splits <= kMaxMlpCtas CTAs, each [hidden x 256] fp32 (+ one chunk of slack per split row)
     const size_t d_pad = (size_t)((max_d + kFeatChunk - 1) / kFeatChunk * kFeatChunk);
     const size_t n_chunks = d_pad / kFeatChunk;
@@ -665,6 +822,18 @@ aa_status launch_assistant_step_mlp(aa_ctx_impl* c, const MlpFeat& f, float* W1_
     while (splits > 1 && (size_t)splits * (size_t)f.hidden * (size_t)p.d_pad * 4 > c->mlp_part_bytes) --splits;
     if ((size_t)splits * (size_t)f.hidden * (size_t)p.d_pad * 4 > c->mlp_part_bytes) return AA_ERR_WORKSPACE;
     p.splits = (int)splits;
+    // The screening's scores and gates stand in for the forward pass when they are the ones of these rows under these
+    // weights: the caller passed scores, the last two-layer screening on this context ran on this very pool (no candidate
+    // list) with this W1, and no update has gone through the context since.
+    const bool scored = c->step_score && c->mlp_gate_cand && c->gate_feat == f.x && c->gate_w1 == f.W1_bf16 && c->gate_n == f.n &&
+                        n_stored == f.n && f.d % 128 == 0 && (uintptr_t)W1_master % 16 == 0;
+    c->gate_feat = nullptr;      // the parameters change below: the gates in the workspace go stale
+    if (scored) {
+        p.score = c->step_score;
+        p.gate_cand = c->mlp_gate_cand;
+        p.gw2_part = reinterpret_cast<float*>(reinterpret_cast<char*>(c->mlp_small) + kSmallBytes);
+        p.gw2_segs = (int)(f.d / 128);
+    }
 
     alignas(64) CUtensorMap map_x, map_w, map_xg;
     if (!encode_bf16_tile_map(&map_x, f.x, (uint64_t)f.n, (uint64_t)f.d, (uint64_t)f.row_stride, gather ? 1 : kHalfRows) ||
@@ -681,8 +850,17 @@ aa_status launch_assistant_step_mlp(aa_ctx_impl* c, const MlpFeat& f, float* W1_
         const int64_t tiles = (m_host + kHalfRows - 1) / kHalfRows;
         int grid = max_ctas;
         if (grid > tiles) grid = (int)tiles;
-        void* args[] = {&map_x, &map_w, &p};
-        if (cudaLaunchKernel(kernel, dim3(grid), dim3(kStepMlpThreads), args, smem, c->stream) != cudaSuccess) return AA_ERR_CUDA;
+        if (scored) {
+            const int64_t groups = (m_host + kRowSlice - 1) / kRowSlice * (kRowSlice / 32);
+            grid = max_ctas;
+            if (grid > (groups + kPrepWarps - 1) / kPrepWarps) grid = (int)((groups + kPrepWarps - 1) / kPrepWarps);
+            void* args[] = {&p};
+            if (cudaLaunchKernel((const void*)mlp_prepare_kernel, dim3(grid), dim3(kPrepThreads), args, 0, c->stream) != cudaSuccess)
+                return AA_ERR_CUDA;
+        } else {
+            void* args[] = {&map_x, &map_w, &p};
+            if (cudaLaunchKernel(kernel, dim3(grid), dim3(kStepMlpThreads), args, smem, c->stream) != cudaSuccess) return AA_ERR_CUDA;
+        }
         ++c->launches;
         // 2. G = P^T X
         const size_t smem2 = 1024 + (size_t)kXStages * kXStageBytes + (size_t)kATiles * kATileBytes + sizeof(GradPipe) + 64;

@@ -183,7 +183,10 @@ def test_mlp_assistant_step_many_tiles_per_cta_and_every_split(aa):
     check_mlp_step(aa, 65536, 40000, 3072, 256, True, None, 0.01)
 
 
-def check_mlp_step(aa, n, m, d, hidden, use_rows, thr, lr):
+def check_mlp_step(aa, n, m, d, hidden, use_rows, thr, lr, scored=None):
+    """scored: None = the step evaluates the forward pass itself; "screen" = the pool is screened first on the same context
+    and the step gets that screening's scores; "altered" = as "screen", but the scores are changed on the way (the oracle
+    gets the same changed scores: the step must really be using what it is handed)."""
     rng = np.random.default_rng(n + d)
     x = W.normal((n, d), 1.0, 60 + d, torch.bfloat16, DEV)
     W1, W1b, b1, w2, b2 = make_mlp(d, hidden, 61 + d)
@@ -196,18 +199,32 @@ def check_mlp_step(aa, n, m, d, hidden, use_rows, thr, lr):
     W1b_before = W1b.clone()
     feat = B.dense_features(x, row_idx=rows_t) if use_rows else B.dense_features(x[:m])
     cnt = torch.tensor([m], dtype=torch.int32, device=DEV)
-    aa.aa_assistant_step(feat, loss, B.mlp_assistant(W1, W1b, b1, w2, b2), lr, threshold=thr, count_dev=cnt)
+    s_given = None
+    if scored is None:
+        aa.aa_assistant_step(feat, loss, B.mlp_assistant(W1, W1b, b1, w2, b2), lr, threshold=thr, count_dev=cnt)
+    else:
+        assert use_rows or m == n                        # the scores are those of the pool's stored rows
+        sink_idx = torch.zeros(n, dtype=torch.int32, device=DEV)
+        sink_cnt = torch.zeros(1, dtype=torch.int32, device=DEV)
+        score = torch.zeros(n, dtype=torch.float32, device=DEV)
+        asst = B.mlp_assistant(W1, W1b, b1, w2, b2)
+        aa.aa_score_shrink(B.dense_features(x), asst, 0.3, 5, 1, sink_idx, sink_cnt, score)
+        if scored == "altered":
+            score = (score * 0.5 + 0.3).contiguous()
+            s_given = score.cpu().numpy().astype(np.float64)
+            s_given = s_given[rows] if use_rows else s_given
+        aa.aa_assistant_step_scored(feat, loss, score, asst, lr, threshold=thr, count_dev=cnt)
     torch.cuda.synchronize()
     assert aa.aa_device_status() == B.AA_OK
     ref = O.assistant_step_mlp(W.to_oracle(x), loss.cpu().numpy(), host["W1"], W1b_bits, host["b1"], host["w2"], b2_0, lr,
-                               T=thr, row_idx=rows)
+                               T=thr, row_idx=rows, s=s_given)
     # The gate [a > 0] is a decision that floating point takes: fp32 accumulation on the GPU, fp64 in the oracle.  Where the
     # oracle's pre-activation lies within the score tolerance of zero (1e-5 of the scale of its terms) either decision is
     # valid, and the W1 gradient may differ by that row's whole contribution; everywhere else the updated W1 is held to the
     # plain bar.  r enters the contraction as two bf16 terms (relative error 2^-17 of each row's contribution).
     gW1 = ref["grads"][0]
     xs = bf16_values(x[:m] if rows is None else x[rows_t.long()])
-    r = O.sigmoid(ref["s"]) - ref["z"]
+    r = O.sigmoid(ref["s"] if s_given is None else s_given) - ref["z"]
     on = ref["a"] > 0
     W1v = bf16_values(W1b_before)
     a_scale = np.abs(host["b1"].astype(np.float64))[None, :] + np.linalg.norm(xs, axis=1)[:, None] * np.linalg.norm(W1v, axis=1)[None, :]
@@ -229,6 +246,77 @@ def check_mlp_step(aa, n, m, d, hidden, use_rows, thr, lr):
     ulp = np.abs(host["W1"]) * 2.0 ** -23 / lr
     fp32 = 1e-6 * (np.abs(r)[:, None] * on).T @ np.abs(xs) * np.abs(w2h)[:, None] / m     # fp32 accumulation over the batch rows
     assert np.all(np.abs(g_gpu - gW1) <= bound + fp32 + 2 * ulp + 1e-12), float(np.max(np.abs(g_gpu - gW1) - bound - fp32 - 2 * ulp))
+
+
+@pytest.mark.parametrize("scored", ["screen", "altered"])
+@pytest.mark.parametrize("n,m,d,hidden,use_rows,thr,lr", [
+    (2000, 1500, 256, 64, True, None, 0.1), (1000, 1000, 384, 256, False, 1.5, 0.1), (5000, 2777, 3072, 256, True, None, 0.05),
+    (700, 1, 128, 32, True, None, 0.1), (1300, 1300, 640, 128, False, None, 1.0), (900, 333, 128, 16, True, None, 0.1),
+])
+def test_mlp_assistant_step_on_the_scores_and_gates_of_the_screening(aa, n, m, d, hidden, use_rows, thr, lr, scored):
+    """The update right after a screening on the same context: r from the screening's scores, the gates [a > 0] from
+    the bits it left in the workspace, grad w2 through  sum_k W1b_uk G_uk + b1_u sum_i r_i [a_iu > 0].  Same bars as the
+    step that evaluates the forward pass itself."""
+    check_mlp_step(aa, n, m, d, hidden, use_rows, thr, lr, scored=scored)
+
+
+def test_mlp_scored_step_many_rows(aa):
+    check_mlp_step(aa, 65536, 40000, 3072, 256, True, None, 0.01, scored="screen")
+
+
+def test_mlp_scored_step_falls_back_when_the_gates_are_not_those_of_the_pool(aa):
+    """Scores are only trusted together with the gates of the same screening.  After an update (the gates are stale), for
+    other weights or another pool the step evaluates the forward pass itself, bit for bit like aa_assistant_step, and
+    never reads the scores."""
+    n, d, hidden, lr = 3000, 256, 64, 0.1
+    x = W.normal((n, d), 1.0, 71, torch.bfloat16, DEV)
+    loss = (W.normal((n,), 1.0, 72, torch.float32, DEV).abs() * 2).contiguous()
+    rows_t = torch.arange(0, n, 2, dtype=torch.int32, device=DEV)
+    cnt = torch.tensor([rows_t.numel()], dtype=torch.int32, device=DEV)
+    garbage = torch.full((n,), float("nan"), dtype=torch.float32, device=DEV)
+    sink_idx = torch.zeros(n, dtype=torch.int32, device=DEV)
+    sink_cnt = torch.zeros(1, dtype=torch.int32, device=DEV)
+    score = torch.zeros(n, dtype=torch.float32, device=DEV)
+    feat = B.dense_features(x, row_idx=rows_t)
+
+    def fresh():
+        return [t.clone() for t in make_mlp(d, hidden, 73)]
+
+    def plain_steps(k):
+        p = fresh()
+        for _ in range(k):
+            aa.aa_assistant_step(feat, loss, B.mlp_assistant(*p), lr, count_dev=cnt)
+        torch.cuda.synchronize()
+        return p
+
+    # (a) a second scored step without a screening in between: the first one has changed the parameters
+    p = fresh()
+    aa.aa_score_shrink(B.dense_features(x), B.mlp_assistant(*p), 0.3, 5, 1, sink_idx, sink_cnt, score)
+    aa.aa_assistant_step_scored(feat, loss, score, B.mlp_assistant(*p), lr, count_dev=cnt)
+    torch.cuda.synchronize()
+    after_one = [t.clone() for t in p]
+    aa.aa_assistant_step_scored(feat, loss, garbage, B.mlp_assistant(*p), lr, count_dev=cnt)
+    torch.cuda.synchronize()
+    q = [t.clone() for t in after_one]
+    aa.aa_assistant_step(feat, loss, B.mlp_assistant(*q), lr, count_dev=cnt)
+    torch.cuda.synchronize()
+    for got, want in zip(p, q):
+        assert torch.equal(got, want)
+    # (b) weights other than the ones the pool was screened with
+    p, other = fresh(), fresh()
+    aa.aa_score_shrink(B.dense_features(x), B.mlp_assistant(*p), 0.3, 5, 1, sink_idx, sink_cnt, score)
+    aa.aa_assistant_step_scored(feat, loss, garbage, B.mlp_assistant(*other), lr, count_dev=cnt)
+    torch.cuda.synchronize()
+    for got, want in zip(other, plain_steps(1)):
+        assert torch.equal(got, want)
+    # (c) a screening with a candidate list leaves no usable gates
+    p = fresh()
+    aa.aa_score_shrink(B.dense_features(x, row_idx=rows_t), B.mlp_assistant(*p), 0.3, 5, 1, sink_idx, sink_cnt, score)
+    aa.aa_assistant_step_scored(feat, loss, garbage, B.mlp_assistant(*p), lr, count_dev=cnt)
+    torch.cuda.synchronize()
+    for got, want in zip(p, plain_steps(1)):
+        assert torch.equal(got, want)
+    assert aa.aa_device_status() == B.AA_OK
 
 
 def test_mlp_step_empty_batch_and_zero_lr(aa):
