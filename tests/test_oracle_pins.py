@@ -596,6 +596,36 @@ def test_composed_mlp_step_descends_the_objective_to_first_order():
     assert np.array_equal(out["z"], z)
 
 
+def test_mlp_step_with_given_scores_and_the_grad_w2_identity():
+    """(1) Handing assistant_step_mlp its own pre-activations changes nothing; handing it other ones changes r only:
+    with s = +/- large the residual is 1 - z or -z and grad b2 has the closed form (count of z = 0) / M resp. -(count of z = 1) / M.
+    (2) relu(a) = [a > 0] (W1 . x + b1) ties the oracle's four gradients together:
+    w2_u grad_w2_u ... = sum_k W1_uk gW1_uk + b1_u gb1_u  (both sides are w2_u sum_i r_i relu(a_iu) / M)."""
+    rng = np.random.default_rng(12)
+    n, d, hidden = 60, 7, 6
+    x = rng.normal(size=(n, d)).astype(np.float32)
+    W1 = (rng.integers(-32, 32, size=(hidden, d)) / 16.0).astype(np.float32)
+    W1_bits = O.round_bf16(W1)
+    b1 = (rng.normal(size=hidden) * 0.3).astype(np.float32)
+    w2 = rng.normal(size=hidden).astype(np.float32)
+    b2 = np.float32(-0.1)
+    f = np.abs(rng.normal(size=n)).astype(np.float32)
+    base = O.assistant_step_mlp(x, f, W1, W1_bits, b1, w2, b2, 0.1)
+    same = O.assistant_step_mlp(x, f, W1, W1_bits, b1, w2, b2, 0.1, s=base["s"])
+    for key in ("W1", "b1", "w2", "b2"):
+        assert np.array_equal(np.asarray(base[key]), np.asarray(same[key]))
+    z = base["z"]
+    hi = O.assistant_step_mlp(x, f, W1, W1_bits, b1, w2, b2, 0.1, s=np.full(n, 60.0))
+    lo = O.assistant_step_mlp(x, f, W1, W1_bits, b1, w2, b2, 0.1, s=np.full(n, -60.0))
+    assert abs(hi["grads"][3] - float(np.sum(z == 0)) / n) < 1e-12
+    assert abs(lo["grads"][3] + float(np.sum(z == 1)) / n) < 1e-12
+    gW1, gb1, gw2, gb2 = base["grads"]
+    lhs = w2.astype(np.float64) * gw2
+    rhs = np.sum(W1.astype(np.float64) * gW1, axis=1) + b1.astype(np.float64) * gb1
+    assert np.allclose(lhs, rhs, rtol=1e-12, atol=1e-14)
+    assert np.abs(lhs).max() > 1e-3
+
+
 def test_batch_cut_is_the_literal_walk_of_algorithm_1():
     """batch_cut on the ordered survivors equals the sequential Algorithm 1 loop (batch and candidates consumed), and the
     token-budget form has the closed forms of unit lengths and of a budget nothing fits in."""
