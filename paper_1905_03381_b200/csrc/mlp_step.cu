@@ -286,13 +286,29 @@ mlp_residual_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
 }
 
 // ---------------------------------------------------------------- residuals from the screening's scores and gates
-constexpr int kPrepThreads = 1024;
+constexpr int kPrepThreads = 512;
 constexpr int kPrepWarps = kPrepThreads / 32;
+
+// Transpose of a 32 x 32 bit matrix held one row per lane (bit c of lane i's word = element [i][c]): five rounds of
+// block swaps between lanes j apart.  Afterwards bit i of lane c's word is element [i][c].
+__device__ __forceinline__ uint32_t warp_bit_transpose(uint32_t x, int lane) {
+    const uint32_t masks[5] = {0x0000FFFFu, 0x00FF00FFu, 0x0F0F0F0Fu, 0x33333333u, 0x55555555u};
+#pragma unroll
+    for (int step = 0; step < 5; ++step) {
+        const int j = 16 >> step;
+        const uint32_t m = masks[step];
+        const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, x, j);
+        // lanes with bit j clear keep their low blocks and take the partner's low blocks into their high ones;
+        // the partner does the opposite
+        x = (lane & j) ? ((x & ~m) | ((other >> j) & m)) : ((x & m) | ((other & m) << j));
+    }
+    return x;
+}
 
 __global__ void __launch_bounds__(kPrepThreads, 1) mlp_prepare_kernel(MlpStepParams p) {
     __shared__ double red[kPrepWarps];
     __shared__ float col_s[kPrepWarps][kMaxHidden];      // per warp: sum_i r_i [a_iu > 0]
-    __shared__ float r_s[kPrepWarps][32];
+    __shared__ float tab_s[kPrepWarps][8][16];           // per warp: sums of r over every subset of each 4-row group
     __shared__ float rsum_s[kPrepWarps];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int64_t m = mlp_batch_size(p);
@@ -351,25 +367,32 @@ __global__ void __launch_bounds__(kPrepThreads, 1) mlp_prepare_kernel(MlpStepPar
             p.r_hi[i] = hi;
             p.r_lo[i] = __float2bfloat16_rn(r - __bfloat162float(hi));
         }
-        __syncwarp();
-        r_s[warp][lane] = r;
-        __syncwarp();
+        // Table for the column sums: entry [k][s] = sum of r over the rows 4 k + b of this group whose bit b is set in s.
+        // Lane l fills the four entries [l >> 2][4 (l & 3) .. + 3].
+        {
+            const int k = lane >> 2;
+            const float r0 = __shfl_sync(0xFFFFFFFFu, r, 4 * k), r1 = __shfl_sync(0xFFFFFFFFu, r, 4 * k + 1);
+            const float r2 = __shfl_sync(0xFFFFFFFFu, r, 4 * k + 2), r3 = __shfl_sync(0xFFFFFFFFu, r, 4 * k + 3);
+            const float high = ((lane & 1) ? r2 : 0.0f) + ((lane & 2) ? r3 : 0.0f);      // bits 2 and 3 of s = lane & 3
+            __syncwarp();                                   // the previous group's look-ups are done
+            float* t = &tab_s[warp][k][4 * (lane & 3)];
+            t[0] = high;
+            t[1] = r0 + high;
+            t[2] = r1 + high;
+            t[3] = (r0 + r1) + high;
+            __syncwarp();
+        }
         const uint32_t words[kMaxHidden / 32] = {g_lo.x, g_lo.y, g_lo.z, g_lo.w, g_hi.x, g_hi.y, g_hi.z, g_hi.w};
         uint32_t* gate_dst = p.gate_bits + (g >> 1) * (2 * kMaxHidden) + (g & 1);
 #pragma unroll
         for (int c = 0; c < kMaxHidden / 32; ++c) {
             if (c * 32 < p.g.hidden) {
-                // 32 x 32 bit transpose: lane q ends with unit c * 32 + q over the warp's rows
-                uint32_t mine = 0;
-#pragma unroll
-                for (int q = 0; q < 32; ++q) {
-                    const uint32_t rows_of_unit = __ballot_sync(0xFFFFFFFFu, (words[c] >> q) & 1u);
-                    if (lane == q) mine = rows_of_unit;
-                }
+                // lane q ends with unit c * 32 + q over the warp's rows
+                const uint32_t mine = warp_bit_transpose(words[c], lane);
                 gate_dst[(c * 32 + lane) * 2] = mine;
                 float acc = 0.0f;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) acc += ((mine >> j) & 1u) ? r_s[warp][j] : 0.0f;
+                for (int k = 0; k < 8; ++k) acc += tab_s[warp][k][(mine >> (4 * k)) & 15u];
                 sum_p[c] += acc;
             }
         }
