@@ -12,12 +12,12 @@
 //
 //   warp 0        producer: tickets of 16 batch rows (two stages), one bulk copy per row; publishes which rows a stage
 //                 holds (a running stage count in shared memory) before its copies are issued.
-//   warps 1, 2    the batch-mean threshold (this CTA's share of the loss sum, then every CTA's share in a fixed
-//                 order) and the residuals r_i = sigmoid(score[row_i]) - z_i of a stage; the two warps take alternate
+//   warps 1, 2    the residuals r_i = sigmoid(score[row_i]) - z_i of a stage; the two warps take alternate
 //                 stages (a stage's residuals hang on two dependent loads: batch list entry, then that row's score)
 //                 and are done before the rows land.
-//   warps 3..18   column sums: each owns 12 feature blocks whose accumulator fragments stay in registers for the
-//                 whole kernel.
+//   warps 3..18   first the batch-mean threshold (all M losses, added in a fixed order in every CTA: no CTA waits for
+//                 another), then column sums: each owns 12 feature blocks whose accumulator fragments stay in
+//                 registers for the whole kernel.
 // CTAs write column sums to the partial buffer; once all of them have (a cooperative launch keeps the grid
 // co-resident, the wait is bounded all the same) each CTA adds up a slice of the columns and takes the SGD or Adam
 // step for it, so the step is one launch.
@@ -55,8 +55,8 @@ struct ScoredControl {
     long long first_row[kMMaxStages];
     unsigned int valid[kMMaxStages];
     alignas(16) __nv_bfloat16 r_split[kMMaxStages][3][kMRows];   // hi / mid / lo terms of the residuals
-    uint64_t t_ready;                         // the batch-mean threshold is in T_mean
-    double T_mean;
+    uint64_t t_ready;                         // every column warp's share of the loss sum is in t_part
+    double t_part[kCompWarps];
     float bias_part[kResWarps];
     int published;                            // stage sequence numbers below this have their first_row / valid written
     int stop_j;
@@ -115,7 +115,7 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_scored_kernel(StepPa
             mbar_init(&cb->x_empty[s], kCompWarps);
             mbar_init(&cb->r_ready[s], 1);
         }
-        mbar_init(&cb->t_ready, 1);
+        mbar_init(&cb->t_ready, kCompWarps);
         for (int q = 0; q < kResWarps; ++q) cb->bias_part[q] = 0.0f;
         cb->published = 0;
         cb->stop_j = 0x7FFFFFFF;
@@ -200,56 +200,10 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_scored_kernel(StepPa
     } else if (warp <= kResWarps) {
         const int aw = warp - 1;
         bool ok = true;
-        // ------------------------------------------------------------ threshold (warp 1)
-        // Shrinking threshold T: the caller's value, or the mean of the batch losses.  Summing all M losses in every
-        // CTA costs more than the first ring stages, so each CTA adds one slice (fixed order: lane stride, then a
-        // shuffle tree), publishes its share, and every CTA adds the shares in one fixed order once all are in.
+        // Shrinking threshold T: the caller's value, or the mean of the batch losses.  The sixteen column warps, which
+        // have nothing to do until the first residuals exist, add all M losses in every CTA (a fixed order, so every CTA
+        // and both residual warps arrive at the same bits); no CTA waits for another one.
         const bool mean_T = p.thresh_mode != AA_THRESH_VALUE;
-        if (mean_T && aw == 0) {
-            const int64_t per = ((m + gridDim.x - 1) / gridDim.x + 3) / 4 * 4;
-            const int64_t s_lo = (int64_t)blockIdx.x * per, s_hi = s_lo + per < m ? s_lo + per : m;
-            double acc = 0.0;
-            {
-                float f[8];      // the usual slice is a few hundred losses: eight loads per lane in flight together
-#pragma unroll
-                for (int u = 0; u < 8; ++u) f[u] = s_lo + lane + 32 * u < s_hi ? __ldg(p.loss + s_lo + lane + 32 * u) : 0.0f;
-#pragma unroll
-                for (int u = 0; u < 8; ++u) acc += (double)f[u];
-                for (int64_t i = s_lo + lane + 256; i < s_hi; i += 32) acc += (double)__ldg(p.loss + i);
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-            if (lane == 0) {
-                p.loss_sums[blockIdx.x] = acc;
-                __threadfence();
-                atomicAdd(&p.ctl->sums_in, 1u);
-            }
-            __syncwarp();
-            unsigned int polls = 0;
-            while (*(volatile unsigned int*)&p.ctl->sums_in < gridDim.x && !*abort_flag) {
-                if (++polls > kSpinLimit) break;
-                __nanosleep(32);
-            }
-            if (*(volatile unsigned int*)&p.ctl->sums_in < gridDim.x) {
-                ok = false;
-                if (lane == 0) scored_give_up(p, cb);
-            } else {
-                __threadfence();
-                double share[5];      // lane l adds shares l, l + 32, ... (loads in flight together); then a fixed shuffle tree
-#pragma unroll
-                for (int u = 0; u < 5; ++u) share[u] = lane + 32u * u < gridDim.x ? __ldcg(p.loss_sums + lane + 32 * u) : 0.0;
-                double total = 0.0;
-#pragma unroll
-                for (int u = 0; u < 5; ++u) total += share[u];
-                for (unsigned int q = lane + 160; q < gridDim.x; q += 32) total += __ldcg(p.loss_sums + q);
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xFFFFFFFFu, total, o);
-                if (lane == 0) {
-                    cb->T_mean = m > 0 ? total / (double)m : 0.0;
-                    mbar_arrive(&cb->t_ready);
-                }
-            }
-        }
         {
             // -------------------------------------------------------- residuals: the two warps take alternate stages
             const int n_res = kResWarps;
@@ -271,7 +225,10 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_scored_kernel(StepPa
                 }
                 if (!have_T) {
                     if (!mbar_wait(&cb->t_ready, 0, abort_flag)) { ok = false; break; }
-                    T_shrink = *(volatile double*)&cb->T_mean;
+                    double total = 0.0;
+#pragma unroll
+                    for (int q = 0; q < kCompWarps; ++q) total += *(volatile double*)&cb->t_part[q];
+                    T_shrink = m > 0 ? total / (double)m : 0.0;
                     have_T = true;
                 }
                 if (lane < kMRows) {
@@ -304,6 +261,38 @@ __global__ void __launch_bounds__(kMThreads, 1) linear_grad_scored_kernel(StepPa
         for (int q = 0; q < kMMaxBlocks; ++q)
 #pragma unroll
             for (int e = 0; e < 4; ++e) acc[q][e] = 0.0f;
+        if (p.thresh_mode != AA_THRESH_VALUE) {
+            // this warp's share of the loss sum: elements (or 16-byte groups) cw * 32 + lane, + 512, ...; then a shuffle tree
+            const int ct = cw * 32 + lane;
+            double part = 0.0;
+            if (((uintptr_t)p.loss & 15) == 0) {
+                const int64_t quads = m >> 2;
+                const float4* l4 = reinterpret_cast<const float4*>(p.loss);
+                int64_t q = ct;
+                for (; q + 3 * kCompWarps * 32 < quads; q += 4 * kCompWarps * 32) {        // four loads in flight together
+                    const float4 a = __ldg(l4 + q), b = __ldg(l4 + q + kCompWarps * 32), c4 = __ldg(l4 + q + 2 * kCompWarps * 32),
+                                 d4 = __ldg(l4 + q + 3 * kCompWarps * 32);
+                    part += ((double)a.x + (double)a.y) + ((double)a.z + (double)a.w);
+                    part += ((double)b.x + (double)b.y) + ((double)b.z + (double)b.w);
+                    part += ((double)c4.x + (double)c4.y) + ((double)c4.z + (double)c4.w);
+                    part += ((double)d4.x + (double)d4.y) + ((double)d4.z + (double)d4.w);
+                }
+                for (; q < quads; q += kCompWarps * 32) {
+                    const float4 a = __ldg(l4 + q);
+                    part += ((double)a.x + (double)a.y) + ((double)a.z + (double)a.w);
+                }
+                for (int64_t i = (quads << 2) + ct; i < m; i += kCompWarps * 32) part += (double)__ldg(p.loss + i);
+            } else {
+                for (int64_t i = ct; i < m; i += kCompWarps * 32) part += (double)__ldg(p.loss + i);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
+            if (lane == 0) {
+                cb->t_part[cw] = part;
+                mbar_arrive(&cb->t_ready);
+            }
+            __syncwarp();
+        }
         bool ok = true;
         for (int j = 0; ok; ++j) {
             const int stage = j % S, use = j / S;
