@@ -439,10 +439,9 @@ aa_status launch_assistant_grad_dense_scored(aa_ctx_impl* c, StepParams& p, int*
     int grid = c->sm_count;
     if (grid > n_tickets) grid = (int)n_tickets;
     if (grid < 1) grid = 1;
-    // partial buffer: [grid][d_pad] column sums, [grid] bias sums, then [grid] doubles for the shares of the loss sum
-    const int64_t sums_at = ((int64_t)grid * (p.d_pad + 1) + 1) / 2 * 2;
-    if (sums_at + 2 * (int64_t)grid > c->partial_floats) return AA_ERR_UNSUPPORTED;
-    p.loss_sums = reinterpret_cast<double*>(c->partials + sums_at);
+    // partial buffer: [grid][d_pad] column sums, then [grid] bias sums
+    if ((int64_t)grid * (p.d_pad + 1) > c->partial_floats) return AA_ERR_UNSUPPORTED;
+    p.loss_sums = nullptr;
     const void* kernel = (const void*)linear_grad_scored_kernel;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return AA_ERR_CUDA;
     void* args[] = {&p, &g};
