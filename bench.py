@@ -478,7 +478,7 @@ def leg_mlp(torch, B, W, dev, peaks, small):
 
 def leg_conv(torch, B, W, dev, peaks, small, clocks_mhz):
     """Convolutional Assistant (Boss's 3 x 3 convolution with 16 channels -> rectifier -> 4 x 4 average pooling -> linear
-    layer) on a 65,536-image pool: the feature kernel alone (plain fp32 arithmetic: an ALU roofline), then the screen of
+    layer) on a 65,536-image pool: the feature kernel alone (a small contraction on the warp-level matrix instructions), then the screen of
     the linear layer on the 1024 features per instance."""
     cfg = W.ConvShape()
     if small:
@@ -502,15 +502,27 @@ def leg_conv(torch, B, W, dev, peaks, small, clocks_mhz):
     sm_mhz = clocks_mhz or 1965.0
     alu_peak = 148 * 128 * 2 * sm_mhz * 1e6 / 1e12          # fp32 lanes x 2 flop per multiply-add x SM clock
     ach = flops / (ms_c * 1e-3) / 1e12
+    # The bf16 kernel multiplies on the warp-level matrix instructions: taps padded to whole 16-tap steps, channels to whole
+    # 8-channel tiles, fp32 taps as three bf16 terms.  ncu counts 8 tensor-pipe cycles per m16n8k16 per SM sub-partition,
+    # i.e. 4096 flop / 8 cycles x 4 sub-partitions x 148 SMs x clock for this instruction path.
+    taps = cfg.c_in * cfg.ksize * cfg.ksize
+    issued = 2.0 * cfg.n * cfg.height * cfg.width * (-(-taps // 16) * 16) * (-(-cfg.c_out // 8) * 8) * 3
+    mma_peak = 148 * 4 * (4096 / 8.0) * sm_mhz * 1e6 / 1e12
+    ach_issued = issued / (ms_c * 1e-3) / 1e12
     out = {
         "workload": f"{cfg.n} images of {cfg.c_in} x {cfg.height} x {cfg.width} bf16 U[0,1), {cfg.c_out} channels of "
                     f"{cfg.ksize} x {cfg.ksize} taps, {cfg.pool} x {cfg.pool} average pooling -> {F} fp32 features per instance",
         "features": {"value": cfg.n / (ms_c * 1e-3), "unit": UNIT, "ms_per_call": ms_c,
-                     "roofline": {"bound": "alu", "kernel": "conv_pool_features_kernel", "achieved": ach, "peak": alu_peak,
-                                  "unit": "TFLOP/s", "frac": ach / alu_peak,
-                                  "peak_kind": f"148 SMs x 128 fp32 lanes x 2 flop x {sm_mhz:.0f} MHz (the sampled SM clock)",
-                                  "flops_per_launch": flops, "avg_launch_ms": ms_c, "best_launch_ms": best_c, "launches_timed": calls_c,
-                                  "hbm_GBs": cfg.n * (cfg.d * 2 + F * 4) / (ms_c * 1e-3) / 1e9}},
+                     "roofline": {"bound": "tensor", "kernel": "conv_pool_mma_kernel", "achieved": ach_issued, "peak": mma_peak,
+                                  "unit": "TFLOP/s", "frac": ach_issued / mma_peak,
+                                  "peak_kind": f"mma.sync m16n8k16 bf16 path: 148 SMs x 4 sub-partitions x 512 flop per cycle x "
+                                               f"{sm_mhz:.0f} MHz (8 tensor-pipe cycles per instruction, from ncu); issued flops "
+                                               f"= 3 bf16 terms of the fp32 taps, taps padded to 16s, channels to 8s",
+                                  "flops_per_launch": issued, "useful_flops_per_launch": flops, "useful_TFLOPs": ach,
+                                  "useful_over_fp32_alu_peak": ach / alu_peak, "fp32_alu_peak_TFLOPs": alu_peak,
+                                  "avg_launch_ms": ms_c, "best_launch_ms": best_c, "launches_timed": calls_c,
+                                  "hbm_GBs": cfg.n * (cfg.d * 2 + F * 4) / (ms_c * 1e-3) / 1e9,
+                                  "hbm_frac": cfg.n * (cfg.d * 2 + F * 4) / (ms_c * 1e-3) / 1e9 / peaks["hbm"]}},
         "linear_layer_screen": {"value": cfg.n / (ms_s * 1e-3), "unit": UNIT, "ms_per_call": ms_s, "accepted": int(cnt.item()),
                                 "roofline": hbm_roofline(cfg.n * F * 4 + F * 4 + 4 * int(cnt.item()), ms_s, best_s, calls_s, peaks,
                                                          kernel="score_shrink_tma_kernel<float>")},

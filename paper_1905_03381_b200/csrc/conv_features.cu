@@ -227,9 +227,17 @@ __global__ void __launch_bounds__(kConvThreads) conv_pool_features_kernel(ConvPa
 
 }  // namespace
 
+// bf16 images of the common shapes go to the matrix-instruction kernel (conv_features_mma.cu)
+aa_status launch_conv_pool_features_mma(aa_ctx_impl* c, const void* x, int dtype, int64_t n, int64_t row_stride, const aa_conv& cv,
+                                        float* phi, int64_t phi_stride);
+
 aa_status launch_conv_pool_features(aa_ctx_impl* c, const void* x, int dtype, int64_t n, int64_t row_stride, const aa_conv& cv,
                                     float* phi, int64_t phi_stride) {
     if (cv.ksize != 1 && cv.ksize != 3 && cv.ksize != 5) return AA_ERR_UNSUPPORTED;
+    {
+        const aa_status st = launch_conv_pool_features_mma(c, x, dtype, n, row_stride, cv, phi, phi_stride);
+        if (st != AA_ERR_UNSUPPORTED) return st;
+    }
     ConvParams p;
     p.x = x;
     p.n = n;

@@ -42,6 +42,11 @@ def features(aa, x, weight, bias, H, Wd, pool):
     (37, 3, 32, 32, 16, 3, 4, torch.bfloat16, 0), (5, 3, 32, 32, 16, 3, 32, torch.bfloat16, 0), (9, 1, 28, 28, 8, 5, 2, torch.float32, 0),
     (20, 3, 12, 12, 5, 3, 1, torch.float32, 4), (3, 2, 8, 24, 7, 1, 8, torch.bfloat16, 8), (300, 3, 32, 32, 16, 3, 8, torch.bfloat16, 0),
     (1, 3, 32, 32, 32, 3, 2, torch.float32, 0),
+    # bf16 shapes of the matrix-instruction kernel: one and two k-steps, one and two channel tiles, every pooling side,
+    # 1 x 1 / 3 x 3 / 5 x 5 windows, padded rows, channel counts that are not a multiple of 8
+    (33, 3, 32, 32, 16, 3, 1, torch.bfloat16, 0), (21, 3, 32, 32, 16, 3, 2, torch.bfloat16, 8), (18, 3, 32, 32, 16, 3, 16, torch.bfloat16, 0),
+    (40, 1, 16, 48, 5, 3, 4, torch.bfloat16, 0), (12, 1, 20, 16, 8, 5, 2, torch.bfloat16, 0), (7, 3, 8, 64, 13, 1, 8, torch.bfloat16, 16),
+    (700, 3, 32, 32, 16, 3, 4, torch.bfloat16, 0),
 ])
 def test_conv_pool_features_match_the_oracle(aa, n, c_in, H, Wd, c_out, k, pool, dtype, pad):
     d = c_in * H * Wd
