@@ -6,7 +6,8 @@
 // (27 for a 3 x 3 window over 3 planes) and up to 16 channels.  A warp takes 16 adjacent pixels of an image row at a time,
 // as two products of shape 16 channels x 8 pixels x 16 taps (mma.sync.m16n8k16, fp32 accumulation):
 //   left operand  (16 channels x 16 taps): the taps, fp32 split into three bf16 terms hi + mid + lo (exact: 3 x 8
-//                 significant bits), held in registers for the whole kernel; the three products go into one accumulator
+//                 significant bits), held in registers for the whole kernel; the three products go into one accumulator (which starts from zero: the bias
+//                 enters with the rectifier, max(a, 0) = max(a - bias, -bias) + bias)
 //   right operand (16 taps x 8 pixels): one ldmatrix.x2.trans.  Row k of that matrix is tap k's view of the 8 pixels:
 //                 8 adjacent elements of the image in shared memory, starting dx elements to the right of the pixels.
 //                 ldmatrix wants every row 16-byte aligned, so the image is kept k times, copy dx shifted left by dx
@@ -67,12 +68,11 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-// the same with the addend given apart from the result (the first product of an accumulator starts from the bias:
-// fragment entries 0, 1 belong to channel g, entries 2, 3 to channel g + 8)
-__device__ __forceinline__ void mma_bf16_16816_from(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1, float c_lo, float c_hi) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%10, %10, %11, %11};"
+// the first product of an accumulator: no addend
+__device__ __forceinline__ void mma_bf16_16816_first(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%10, %10, %10, %10};"
                  : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(c_lo), "f"(c_hi));
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.0f));
 }
 // Two 8 x 8 matrices of 16-bit elements, transposed on the way: lanes 0..7 give the row addresses of the first matrix,
 // lanes 8..15 those of the second (16-byte aligned); lane (g, t) receives elements [2t][g], [2t + 1][g] of each.
@@ -133,6 +133,7 @@ __global__ void __launch_bounds__(kCmThreads, 5) conv_pool_mma_kernel(ConvMmaPar
     }
     const float b_lo = (p.bias && g < p.c_out) ? __ldg(p.bias + g) : 0.0f;
     const float b_hi = (p.bias && g + 8 < p.c_out) ? __ldg(p.bias + g + 8) : 0.0f;
+    const float nb_lo = -b_lo, nb_hi = -b_hi;
 
     const int strips = p.width >> 4;
     const int ph = p.height / p.pool, pw = p.width / p.pool;
@@ -198,14 +199,29 @@ __global__ void __launch_bounds__(kCmThreads, 5) conv_pool_mma_kernel(ConvMmaPar
                     for (int tr = 0; tr < 3; ++tr)
 #pragma unroll
                         for (int tile = 0; tile < 2; ++tile) {
-                            if (ks == 0 && tr == 0) mma_bf16_16816_from(c[tile], aw[ks][tr], b[tile][ks][0], b[tile][ks][1], b_lo, b_hi);
+                            if (ks == 0 && tr == 0) mma_bf16_16816_first(c[tile], aw[ks][tr], b[tile][ks][0], b[tile][ks][1]);
                             else mma_bf16_16816(c[tile], aw[ks][tr], b[tile][ks][0], b[tile][ks][1]);
                         }
-                // rectifier and the vertical part of the window
+                // rectifier and the vertical part of the window.  The accumulators hold a - bias: max(a, 0) = max(a - bias, -bias)
+                // + bias, and the bias goes in once per window below.
 #pragma unroll
-                for (int tile = 0; tile < 2; ++tile)
+                for (int tile = 0; tile < 2; ++tile) {
+                    vacc[tile][0] += fmaxf(c[tile][0], nb_lo);
+                    vacc[tile][1] += fmaxf(c[tile][1], nb_lo);
+                    vacc[tile][2] += fmaxf(c[tile][2], nb_hi);
+                    vacc[tile][3] += fmaxf(c[tile][3], nb_hi);
+                }
+            }
+            {
+                // every entry has added up `pool` rows
+                const float rows = (float)p.pool;
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) vacc[tile][e] += fmaxf(c[tile][e], 0.0f);
+                for (int tile = 0; tile < 2; ++tile) {
+                    vacc[tile][0] = fmaf(rows, b_lo, vacc[tile][0]);
+                    vacc[tile][1] = fmaf(rows, b_lo, vacc[tile][1]);
+                    vacc[tile][2] = fmaf(rows, b_hi, vacc[tile][2]);
+                    vacc[tile][3] = fmaf(rows, b_hi, vacc[tile][3]);
+                }
             }
             // The horizontal part.  Entries 0, 1 of a fragment: channel g, pixels 2t, 2t + 1 of the tile; entries 2, 3:
             // channel g + 8, the same pixels.
