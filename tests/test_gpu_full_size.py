@@ -217,3 +217,68 @@ def test_mlp_shape_loss_and_step_full_size():
         # both sides round P to bf16 identically (same rows, same parameters); what differs is the fp32 summation order
         assert float((f_ - p_).abs().max()) <= 2e-4 * scale, (name, float((f_ - p_).abs().max()), scale)
     aa.close()
+
+
+def test_conv_shape_full_size_sampled():
+    """Convolutional Assistant at the size that is timed (65,536 images of 3 x 32 x 32 bf16, 16 channels of 3 x 3 taps,
+    4 x 4 pooling): the oracle evaluates sampled images; the bar is the one of test_gpu_conv.py."""
+    build.build()
+    cfg = W.ConvShape()
+    x = cfg.pool_images(0, DEV)
+    weight, bias = cfg.conv(DEV)
+    aa = B.AutoAssist(max_rows=cfg.n, max_d=max(cfg.d, cfg.features), device=DEV)
+    phi = torch.full((cfg.n, cfg.features), -9.0, dtype=torch.float32, device=DEV)
+    aa.aa_conv_pool_features(B.dense_features(x), B.conv_layer(weight, bias, cfg.height, cfg.width, cfg.pool), phi)
+    torch.cuda.synchronize()
+    assert aa.aa_device_status() == B.AA_OK
+    sample = sample_rows(cfg.n, 120, 9)
+    xs = rows_of(x, sample).contiguous()
+    ref = O.conv_pool_features(W.to_oracle(xs), cfg.c_in, cfg.height, cfg.width, weight.cpu().numpy(), bias.cpu().numpy(), cfg.pool)
+    scale = O.conv_pool_features(W.to_oracle(xs.abs()), cfg.c_in, cfg.height, cfg.width, weight.abs().cpu().numpy(),
+                                 bias.abs().cpu().numpy(), cfg.pool)
+    got = rows_of(phi, sample).cpu().numpy()
+    err = np.abs(got - ref)
+    assert np.all(err <= 1e-5 * (np.abs(ref) + scale) + 1e-30), float(np.max(err / (np.abs(ref) + scale + 1e-30)))
+    assert float(phi.min()) >= 0.0 and ref.std() > 0.01          # every image was written (rectified values, no -9 left)
+    aa.close()
+
+
+def test_mlp_scored_step_full_size_equals_the_recomputing_step():
+    """Two-layer Assistant at the size that is timed (262,144 x 3072 pool, hidden 256): the update that takes the
+    screening's scores and gate bits must give the parameters of the update that evaluates the forward pass itself, on
+    the batch the screening produced.  Both routes are tied to the oracle at 40,000 rows in test_gpu_mlp.py; here the
+    full-size launch geometry of the scored route is tied to the other one."""
+    build.build()
+    cfg = W.MlpShape()
+    x = cfg.pool(DEV)
+    W1, b1, w2, b2 = cfg.assistant(DEV)
+    b1 = W.normal((cfg.hidden,), 0.1, 21, torch.float32, DEV)
+    aa = B.AutoAssist(max_rows=cfg.n, max_d=cfg.d, max_hidden=cfg.hidden, device=DEV)
+    out_idx = torch.zeros(cfg.n, dtype=torch.int32, device=DEV)
+    cnt = torch.zeros(1, dtype=torch.int32, device=DEV)
+    score = torch.zeros(cfg.n, dtype=torch.float32, device=DEV)
+    loss = (W.normal((cfg.n,), 1.0, 22, torch.float32, DEV).abs() * 2).contiguous()
+    feat, batch = B.dense_features(x), B.dense_features(x, row_idx=out_idx)
+
+    def fresh():
+        return [W1.clone(), W1.to(torch.bfloat16).contiguous(), b1.clone(), w2.clone(), b2.clone()]
+
+    P = fresh()
+    aa.aa_score_shrink(feat, B.mlp_assistant(*P), cfg.gamma, cfg.philox_seed, 2, out_idx, cnt, score)
+    aa.aa_assistant_step_scored(batch, loss, score, B.mlp_assistant(*P), 0.5, count_dev=cnt)
+    Q = fresh()
+    aa.aa_assistant_step(batch, loss, B.mlp_assistant(*Q), 0.5, count_dev=cnt)
+    torch.cuda.synchronize()
+    assert aa.aa_device_status() == B.AA_OK
+    m = int(cnt.item())
+    assert 100000 < m < cfg.n
+    start = fresh()
+    for name, got, want, was in zip(("W1", "W1_bf16", "b1", "w2", "b2"), P, Q, start):
+        step = (want.double() - was.double())
+        scale = float(step.abs().max())
+        assert scale > 0, name
+        # the same rows, gates and residuals on both routes; what differs is fp32 summation order (and, for w2, the
+        # identity that takes sum_i r_i relu(a_iu) from the W1-gradient contraction)
+        tol = 2e-4 * scale if name != "W1_bf16" else 2.0 ** -7 * float(want.double().abs().max())
+        assert float((got.double() - want.double()).abs().max()) <= tol, (name, float((got.double() - want.double()).abs().max()), scale)
+    aa.close()
